@@ -1,0 +1,159 @@
+/*
+ * wf_encoder.h -- C ABI of the ragged, hush-terminated speech-encoder library (sm_100a).
+ *
+ * The library implements the encoding stage of a streaming speech pipeline in which each
+ * audio buffer x is followed by a short fixed "hush" segment h instead of being padded to
+ * 30 s (paper Sec. 4.1.2, "New paradigm: hush word": x (+) h), so that the encoder --
+ * the 1,500-token, tens-of-layers cost named in Sec. 1.1 and Sec. 2.3 -- runs over real
+ * tokens only.  Buffers of different lengths are batched without padding (the
+ * variable-length batching problem raised in Sec. 3.3): every activation is a packed
+ * [sum of rows, channels] matrix plus prefix sums.
+ *
+ * Conventions
+ *   - "dev" pointers are CUDA device pointers on the device that was current when the
+ *     encoder was created; "host" pointers are ordinary host memory.
+ *   - All work is enqueued on the `stream` argument (a cudaStream_t passed as void*;
+ *     NULL = the legacy default stream).  Calls return without synchronising unless stated.
+ *     Host arrays are read or written before the call returns.
+ *   - The caller owns every buffer it passes.  The library owns its converted weights,
+ *     tables and workspace, sized at create time and released by wf_encoder_destroy.
+ *   - Errors are return codes; nothing aborts.  After a non-zero return the outputs are
+ *     undefined.  wf_last_error gives a human-readable message for the last failure on a
+ *     handle.  A handle is not thread-safe; distinct handles are independent.
+ *   - Row counts: a buffer of L samples has T = floor(L/160) frames (L >= 401 required);
+ *     with the hush segment of H frames it has T' = T + H rows and n = ceil(T'/2) tokens.
+ */
+#ifndef WF_ENCODER_H
+#define WF_ENCODER_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct wf_encoder wf_encoder;
+
+typedef enum {
+  WF_OK = 0,
+  WF_ERR_INVALID_ARG = 1,
+  WF_ERR_TOO_SHORT = 2,      /* a buffer has fewer than 401 samples                        */
+  WF_ERR_TOO_LONG = 3,       /* a sequence would have more than n_ctx tokens               */
+  WF_ERR_CAPACITY = 4,       /* batch, samples or tokens exceed what create() sized        */
+  WF_ERR_CUDA = 5,           /* a CUDA runtime/driver call failed                          */
+  WF_ERR_DEVICE_TIMEOUT = 6, /* a bounded wait inside a kernel gave up                     */
+  WF_ERR_UNSUPPORTED_ARCH = 7,
+  WF_ERR_UNIMPLEMENTED = 8
+} wf_status;
+
+typedef enum { WF_F32 = 0, WF_BF16 = 1 } wf_dtype;
+
+/* Model and capacity description.  d_model / n_head must be 64; d_model and d_mlp multiples
+ * of 128 (d_model <= 1280); n_mel a multiple of 8, at most 128.  dtype selects the arithmetic
+ * of the encoder body: WF_F32 = float32 SIMT kernels, WF_BF16 = bfloat16 tensor-core kernels
+ * with float32 accumulation, float32 residual stream, bfloat16 output.  The front end is
+ * float32 in both. */
+typedef struct {
+  int n_mel, d_model, n_layer, n_head, d_mlp;
+  int n_ctx;          /* most tokens one sequence may have (positions are a closed form)   */
+  int hush_frames;    /* H; 0 = no hush segment (e.g. a 30 s padded run)                    */
+  int dtype;          /* wf_dtype                                                           */
+  int max_batch;      /* most sequences per call                                            */
+  long max_tokens;    /* most tokens per call (sum over sequences)                          */
+  long max_samples;   /* most audio samples per call (sum over sequences), below 2^31       */
+} wf_config;
+
+/* Weights: float32, device memory, read (and converted) once inside wf_encoder_create.
+ * Linear weights are [out, in] row-major, conv kernels [out, in, 3].  The per-layer members
+ * are HOST arrays of n_layer DEVICE pointers.  The key projection has no bias. */
+typedef struct {
+  const float *mel_fb;                 /* [n_mel, 201] non-negative filterbank               */
+  const float *conv1_w, *conv1_b;      /* [d, n_mel, 3], [d]                                 */
+  const float *conv2_w, *conv2_b;      /* [d, d, 3], [d]                                     */
+  const float *const *ln1_g, *const *ln1_b;
+  const float *const *wq, *const *bq, *const *wk, *const *wv, *const *bv;
+  const float *const *wo, *const *bo;
+  const float *const *ln2_g, *const *ln2_b;
+  const float *const *w1, *const *b1;  /* [d_mlp, d], [d_mlp]                                */
+  const float *const *w2, *const *b2;  /* [d, d_mlp], [d]                                    */
+  const float *lnp_g, *lnp_b;          /* final LayerNorm                                    */
+} wf_weights;
+
+/* Builds an encoder on the current device: converts weights to the layouts the kernels
+ * read, builds the windowed-DFT and sinusoid tables on the device, allocates workspace for
+ * the stated capacities.  Synchronises `stream` before returning.  Fails with
+ * WF_ERR_UNSUPPORTED_ARCH on a device that is not compute capability 10.x.
+ * (Operation: the encoder of Sec. 1.1 / Sec. 2.3; weights are caller-provided.) */
+wf_status wf_encoder_create(const wf_config *cfg, const wf_weights *w, void *stream,
+                            wf_encoder **out);
+
+/* Log-mel front end alone (Sec. 4.1.2, "target level": 16 kHz audio -> 100 rows per second):
+ * reflect-padded 400-point periodic-Hann DFT every 160 samples, power, mel projection,
+ * log10 with floor 1e-10, clamp to (per-buffer maximum - 8), (x + 4) / 4.
+ *   audio       dev  float32, the B buffers back to back (sum of lengths samples)
+ *   lengths     host B sample counts
+ *   mel_out     dev  float32 [sum T_i, n_mel], rows of buffer i start at sum_{j<i} T_j
+ *   frames_out  host B frame counts T_i (may be NULL) */
+wf_status wf_logmel(wf_encoder *enc, const float *audio, const long *lengths, int B,
+                    float *mel_out, long *frames_out, void *stream);
+
+/* The whole path: front end, hush rows appended to each buffer's log-mel rows (x (+) h of
+ * Sec. 4.1.2 at the log-mel level), conv stem, sinusoid positions restarting at 0 for every
+ * sequence, n_layer pre-LN blocks whose attention sees one sequence's tokens only, final
+ * LayerNorm.
+ *   hush_mel        dev  float32 [hush_frames, n_mel] in normalised log-mel units;
+ *                        may be NULL iff hush_frames == 0
+ *   hidden_out      dev  [sum n_i, d_model]; float32 for WF_F32, bfloat16 for WF_BF16
+ *   cu_seqlens_out  host B+1 token prefix sums (may be NULL) */
+wf_status wf_encode(wf_encoder *enc, const float *audio, const long *lengths, int B,
+                    const float *hush_mel, void *hidden_out, int *cu_seqlens_out, void *stream);
+
+/* Same as wf_encode but starting from normalised log-mel rows (e.g. from wf_logmel, or a
+ * raw-audio-level hush word already concatenated by the caller with hush_frames == 0).
+ *   mel     dev  float32 [sum T_i, n_mel] packed;   frames  host B row counts T_i >= 1 */
+wf_status wf_encode_mel(wf_encoder *enc, const float *mel, const long *frames, int B,
+                        const float *hush_mel, void *hidden_out, int *cu_seqlens_out,
+                        void *stream);
+
+/* wf_encode with HOST audio and HOST output: copies the samples to a library-owned device
+ * buffer, encodes, copies the hidden states back, and synchronises `stream`.
+ * `audio_host` and `hidden_out_host` should be pinned for the copies to run at full rate. */
+wf_status wf_encode_host(wf_encoder *enc, const float *audio_host, const long *lengths, int B,
+                         const float *hush_mel, void *hidden_out_host, int *cu_seqlens_out,
+                         void *stream);
+
+/* Synchronises `stream` and reports WF_ERR_DEVICE_TIMEOUT if any kernel's bounded wait gave
+ * up since the last check, WF_ERR_CUDA if the stream is in error, else WF_OK. */
+wf_status wf_check(wf_encoder *enc, void *stream);
+
+wf_status wf_encoder_destroy(wf_encoder *enc);
+const char *wf_last_error(const wf_encoder *enc);
+
+/* Per-kernel-class timing.  When enabled, every launch inside wf_encode* is bracketed by
+ * CUDA events on the caller's stream.  wf_profile_read synchronises, then writes for class c
+ * (0 front end, 1 layout/maps, 2 conv stem GEMMs, 3 LayerNorm, 4 block GEMMs, 5 attention)
+ * the number of launches and their summed milliseconds since the last read, and resets. */
+#define WF_N_KERNEL_CLASSES 6
+wf_status wf_profile_enable(wf_encoder *enc, int on);
+wf_status wf_profile_read(wf_encoder *enc, long *launches, double *millis);
+
+/* Component entry points (used by the parity tests and for profiling one kernel alone).
+ *
+ * wf_gemm_bf16: C = epilogue(A W^T + bias) with the tcgen05 kernel the encoder blocks use
+ * (the four GEMMs of a transformer block, Sec. 1.1).  Needs a WF_BF16 encoder.
+ *   A dev bf16 [M, K] row-major, W dev bf16 [N, K] row-major, bias dev float32 [N];
+ *   mode 0: C bf16 [M, N] = acc + bias;  1: C bf16 = gelu(acc + bias);
+ *   mode 2: C float32 [M, N] += acc + bias (residual update in place).
+ *   K and N must be multiples of 8. */
+wf_status wf_gemm_bf16(wf_encoder *enc, const void *A, const void *W, const float *bias, void *C,
+                       long M, int N, int K, int mode, void *stream);
+
+/* wf_attention: non-causal attention over packed tokens, one softmax per (sequence, head)
+ * over that sequence's keys only (no padded token is computed).  qkv dev [M, 3 d_model]
+ * (q | k | v, head h at columns 64 h), out dev [M, d_model]; element type follows the
+ * encoder's dtype.  cu_seqlens host B+1. */
+wf_status wf_attention(wf_encoder *enc, const void *qkv, const int *cu_seqlens, int B, void *out,
+                       void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WF_ENCODER_H */

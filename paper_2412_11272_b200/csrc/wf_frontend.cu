@@ -1,0 +1,303 @@
+// Log-mel front end: tables, framing + windowed DFT (as a folded real GEMM) + mel + log10,
+// per-buffer normalisation, hush append and the padded-row layout the conv stem reads.
+//
+// The front end of Sec. 4.1.2 ("target level": 16 kHz audio -> 100 log-mel rows per second).
+// All arithmetic is float32: the clamp at (max - 8) exposes 80 dB of dynamic range, which
+// bfloat16 products cannot resolve.
+#include "wf_internal.h"
+
+namespace wf {
+
+// ---------------------------------------------------------------------------------------------
+// Tables.  The periodic Hann window is symmetric (w[n] = w[400-n], w[0] = 0), so with
+// e[n] = s[n] + s[400-n], o[n] = s[n] - s[400-n] (n = 1..199), e[200] = s[200]:
+//   Re X[k] =  sum_{n=1}^{200} w[n] cos(2 pi k n / 400) e[n]
+//   Im X[k] = -sum_{n=1}^{199} w[n] sin(2 pi k n / 400) o[n]
+// basis[0][n-1][k] holds the cosine factors, basis[1][n-1][k] the sine factors (row 199 zero).
+__global__ void build_tables_kernel(float* basis, float* pe, int n_ctx, int d) {
+  const long n_basis = 2L * kFold * kBasisCols;
+  const long n_pe = (long)n_ctx * d;
+  for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < n_basis + n_pe;
+       i += (long)gridDim.x * blockDim.x) {
+    if (i < n_basis) {
+      int which = (int)(i / (kFold * kBasisCols));
+      int r = (int)(i % (kFold * kBasisCols));
+      int n = r / kBasisCols + 1;
+      int k = r % kBasisCols;
+      double v = 0.0;
+      if (k < kBins) {
+        double w = 0.5 - 0.5 * cospi(2.0 * n / 400.0);
+        int a = (k * n) % kNFft;  // exact angle reduction
+        if (which == 0) v = w * cospi(2.0 * a / 400.0);
+        else v = (n == kFold) ? 0.0 : w * sinpi(2.0 * a / 400.0);
+      }
+      basis[i] = (float)v;
+    } else {
+      long j = i - n_basis;
+      int p = (int)(j / d), c = (int)(j % d);
+      int half = d / 2;
+      int ch = c < half ? c : c - half;
+      double inv = exp(-log(10000.0) / (half - 1) * ch);
+      double ang = (double)p * inv;
+      pe[j] = (float)(c < half ? sin(ang) : cos(ang));
+    }
+  }
+}
+
+void launch_build_tables(float* dft_basis, float* pe, int n_ctx, int d, cudaStream_t s) {
+  build_tables_kernel<<<296, 256, 0, s>>>(dft_basis, pe, n_ctx, d);
+}
+
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int float_to_ordered(float f) {
+  int i = __float_as_int(f);
+  return i >= 0 ? i : i ^ 0x7FFFFFFF;
+}
+__device__ __forceinline__ float ordered_to_float(int i) {
+  return __int_as_float(i >= 0 ? i : i ^ 0x7FFFFFFF);
+}
+
+__global__ void fill_seq_max_kernel(int* seq_max, int B) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < B) seq_max[i] = (int)0x80000000;
+}
+void launch_fill_seq_max(int* seq_max, int B, cudaStream_t s) {
+  if (B > 0) fill_seq_max_kernel<<<(B + 255) / 256, 256, 0, s>>>(seq_max, B);
+}
+
+// One CTA = 64 consecutive frames of one buffer.  Phase 1 folds the reflected frames into
+// shared memory; phase 2 is the [64 x 200] x [200 x 201] cosine and sine products with an
+// 8-frame x 7-bin register tile per thread; phase 3 squares into shared memory; phase 4 is
+// the mel projection, log10 and the per-buffer running maximum.
+constexpr int kPStride = 204;
+
+__global__ void __launch_bounds__(256) frontend_kernel(
+    const float* __restrict__ audio, const int* __restrict__ meta, MetaLayout ml, int B,
+    const float* __restrict__ basis, const float* __restrict__ fbt, int n_mel,
+    float* __restrict__ logmel, int* __restrict__ seq_max) {
+  extern __shared__ __align__(16) float smem[];
+  float* e_s = smem;                       // [64][200]
+  float* o_s = smem + kFeFrames * kFold;   // [64][200]
+  float* p_s = smem;                       // [64][204] after the DFT
+
+  const int* tile_off = meta + ml.fe_tile_off;
+  int tile = blockIdx.x;
+  int lo = 0, hi = B - 1;
+  while (lo < hi) {  // last sequence whose first tile is <= tile
+    int mid = (lo + hi + 1) >> 1;
+    if (tile_off[mid] <= tile) lo = mid; else hi = mid - 1;
+  }
+  const int seq = lo;
+  const int t0 = (tile - tile_off[seq]) * kFeFrames;
+  const int T = meta[ml.frames + seq];
+  const int s0 = meta[ml.sample_off + seq];
+  const int L = meta[ml.sample_off + seq + 1] - s0;
+  const float* x = audio + s0;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  for (int idx = tid; idx < kFeFrames * kFold; idx += 256) {
+    int f = idx / kFold, n = idx % kFold + 1;
+    int t = t0 + f;
+    float e = 0.f, o = 0.f;
+    if (t < T) {
+      int c = kHop * t;
+      int ia = c - 200 + n, ib = c + 200 - n;
+      if (ia < 0) ia = -ia;
+      if (ia >= L) ia = 2 * (L - 1) - ia;
+      if (ib < 0) ib = -ib;
+      if (ib >= L) ib = 2 * (L - 1) - ib;
+      float a = x[ia];
+      if (n == kFold) { e = a; }
+      else { float b = x[ib]; e = a + b; o = a - b; }
+    }
+    e_s[idx] = e;
+    o_s[idx] = o;
+  }
+  __syncthreads();
+
+  float acc_r[8][7], acc_i[8][7];
+#pragma unroll
+  for (int f = 0; f < 8; ++f)
+#pragma unroll
+    for (int j = 0; j < 7; ++j) { acc_r[f][j] = 0.f; acc_i[f][j] = 0.f; }
+
+  const float* bc = basis + lane;
+  const float* bs = basis + kFold * kBasisCols + lane;
+  const float* er = e_s + warp * 8 * kFold;
+  const float* orow = o_s + warp * 8 * kFold;
+  for (int n4 = 0; n4 < kFold; n4 += 4) {
+    float4 ev[8], ov[8];
+#pragma unroll
+    for (int f = 0; f < 8; ++f) {
+      ev[f] = *reinterpret_cast<const float4*>(er + f * kFold + n4);
+      ov[f] = *reinterpret_cast<const float4*>(orow + f * kFold + n4);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      float c[7], s[7];
+#pragma unroll
+      for (int j = 0; j < 7; ++j) {
+        c[j] = __ldg(bc + (n4 + u) * kBasisCols + 32 * j);
+        s[j] = __ldg(bs + (n4 + u) * kBasisCols + 32 * j);
+      }
+#pragma unroll
+      for (int f = 0; f < 8; ++f) {
+        float e = u == 0 ? ev[f].x : u == 1 ? ev[f].y : u == 2 ? ev[f].z : ev[f].w;
+        float o = u == 0 ? ov[f].x : u == 1 ? ov[f].y : u == 2 ? ov[f].z : ov[f].w;
+#pragma unroll
+        for (int j = 0; j < 7; ++j) {
+          acc_r[f][j] = fmaf(e, c[j], acc_r[f][j]);
+          acc_i[f][j] = fmaf(o, s[j], acc_i[f][j]);
+        }
+      }
+    }
+  }
+  __syncthreads();  // every warp is done with e_s / o_s before p_s overwrites them
+#pragma unroll
+  for (int f = 0; f < 8; ++f)
+#pragma unroll
+    for (int j = 0; j < 7; ++j) {
+      int k = lane + 32 * j;
+      if (k < kBins) p_s[(warp * 8 + f) * kPStride + k] = acc_r[f][j] * acc_r[f][j] + acc_i[f][j] * acc_i[f][j];
+    }
+  __syncwarp();  // a warp only reads back its own 8 rows
+
+  float mel[8][4];
+#pragma unroll
+  for (int f = 0; f < 8; ++f)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) mel[f][j] = 0.f;
+  const float* pr = p_s + warp * 8 * kPStride;
+  for (int k = 0; k < kBins; ++k) {
+    float w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      int m = lane + 32 * j;
+      w[j] = m < n_mel ? __ldg(fbt + k * n_mel + m) : 0.f;
+    }
+#pragma unroll
+    for (int f = 0; f < 8; ++f) {
+      float p = pr[f * kPStride + k];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) mel[f][j] = fmaf(p, w[j], mel[f][j]);
+    }
+  }
+  float mx = -INFINITY;
+  const long frame0 = meta[ml.frame_off + seq];
+#pragma unroll
+  for (int f = 0; f < 8; ++f) {
+    int t = t0 + warp * 8 + f;
+    if (t < T) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int m = lane + 32 * j;
+        if (m < n_mel) {
+          float lg = log10f(fmaxf(mel[f][j], 1e-10f));
+          logmel[(frame0 + t) * n_mel + m] = lg;
+          mx = fmaxf(mx, lg);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if (lane == 0 && mx > -INFINITY) atomicMax(seq_max + seq, float_to_ordered(mx));
+}
+
+void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, int n_tiles,
+                     const float* dft_basis, const float* mel_fb_t, int n_mel, float* logmel,
+                     int* seq_max, cudaStream_t s) {
+  const int smem = (kFeFrames * kPStride > 2 * kFeFrames * kFold ? kFeFrames * kPStride : 2 * kFeFrames * kFold) *
+                   (int)sizeof(float);  // 102,400 B
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(frontend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
+  }
+  if (n_tiles > 0)
+    frontend_kernel<<<n_tiles, 256, smem, s>>>(audio, meta, ml, B, dft_basis, mel_fb_t, n_mel, logmel,
+                                                seq_max);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Normalisation: max(lg, max_i - 8), (x + 4) / 4, written either packed (wf_logmel) or into
+// the padded-row layout with the hush rows behind each buffer's rows (x (+) h at log-mel level).
+// Padded-row layout of sequence i (R_i = 2 (n_i + 1) rows starting at the even row P_i):
+//   row P_i            zero   (left conv padding)
+//   rows P_i+1 ..      T_i audio rows, then H hush rows
+//   remaining 1-2 rows zero   (right conv padding, rounds R_i up to even)
+template <typename OutT>
+__global__ void __launch_bounds__(256) normalise_kernel(
+    const float* __restrict__ logmel, const int* __restrict__ seq_max,
+    const float* __restrict__ mel_in, const int* __restrict__ meta, MetaLayout ml, int n_mel, int dst_ld,
+    int hush_frames, const float* __restrict__ hush, OutT* __restrict__ dst, int mode) {
+  const int seq = blockIdx.y;
+  const int lr = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  const int T = meta[ml.frames + seq];
+  const long frame0 = meta[ml.frame_off + seq];
+  float floor_v = 0.f;
+  if (logmel != nullptr) floor_v = ordered_to_float(seq_max[seq]) - 8.0f;
+  if (mode == 0) {
+    if (lr >= T) return;
+    for (int m = lane; m < n_mel; m += 32) {
+      float v = (fmaxf(logmel[(frame0 + lr) * n_mel + m], floor_v) + 4.0f) * 0.25f;
+      dst[(frame0 + lr) * dst_ld + m] = (OutT)v;
+    }
+    return;
+  }
+  const int p0 = meta[ml.prow_off + seq];
+  const int R = meta[ml.prow_off + seq + 1] - p0;
+  if (lr >= R) return;
+  const int t = lr - 1;
+  for (int m = lane; m < n_mel; m += 32) {
+    float v = 0.f;
+    if (t >= 0 && t < T) {
+      v = mel_in != nullptr ? mel_in[(frame0 + t) * n_mel + m]
+                            : (fmaxf(logmel[(frame0 + t) * n_mel + m], floor_v) + 4.0f) * 0.25f;
+    } else if (t >= T && t < T + hush_frames) {
+      v = hush[(long)(t - T) * n_mel + m];
+    }
+    dst[(long)(p0 + lr) * dst_ld + m] = (OutT)v;
+  }
+}
+
+void launch_normalise(const float* logmel, const int* seq_max, const float* mel_in, const int* meta,
+                      MetaLayout ml, int B, int max_rows, int n_mel, int dst_ld, int hush_frames,
+                      const float* hush, void* dst, int dst_bf16, int mode, cudaStream_t s) {
+  if (B <= 0 || max_rows <= 0) return;
+  dim3 grid((max_rows + 7) / 8, B);
+  if (dst_bf16)
+    normalise_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(logmel, seq_max, mel_in, meta, ml, n_mel, dst_ld,
+                                                         hush_frames, hush, (__nv_bfloat16*)dst, mode);
+  else
+    normalise_kernel<float><<<grid, 256, 0, s>>>(logmel, seq_max, mel_in, meta, ml, n_mel, dst_ld,
+                                                 hush_frames, hush, (float*)dst, mode);
+}
+
+// Row maps for the conv-stem epilogues: which padded rows hold data, and where each stride-2
+// output row lands in the packed token matrix together with its position in its sequence.
+__global__ void build_maps_kernel(const int* __restrict__ meta, MetaLayout ml, int hush_frames,
+                                  int* __restrict__ row_valid, int2* __restrict__ row_dst) {
+  const int seq = blockIdx.y;
+  const int lr = blockIdx.x * blockDim.x + threadIdx.x;
+  const int p0 = meta[ml.prow_off + seq];
+  const int R = meta[ml.prow_off + seq + 1] - p0;
+  if (lr >= R) return;
+  const int rows = meta[ml.frames + seq] + hush_frames;
+  row_valid[p0 + lr] = (lr >= 1 && lr <= rows) ? 1 : 0;
+  if (lr < R / 2) {
+    const int tok0 = meta[ml.tok_off + seq];
+    const int n = meta[ml.tok_off + seq + 1] - tok0;
+    row_dst[p0 / 2 + lr] = make_int2(lr < n ? tok0 + lr : -1, lr);
+  }
+}
+
+void launch_build_maps(const int* meta, MetaLayout ml, int B, int max_rows, int hush_frames,
+                       int* row_valid, int2* row_dst, cudaStream_t s) {
+  if (B <= 0 || max_rows <= 0) return;
+  dim3 grid((max_rows + 255) / 256, B);
+  build_maps_kernel<<<grid, 256, 0, s>>>(meta, ml, hush_frames, row_valid, row_dst);
+}
+
+}  // namespace wf

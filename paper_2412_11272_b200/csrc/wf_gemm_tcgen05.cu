@@ -1,0 +1,313 @@
+// bf16 GEMM for sm_100a: C = epilogue(A W^T), A [M, K] and W [N, K] both K-major.
+//
+// Persistent, warp-specialised CTAs of 192 threads:
+//   warp 0      one lane issues TMA loads (A 128 x 64 and W BN x 64 boxes, 128-byte swizzle)
+//               into a ring of shared-memory stages guarded by full/empty mbarriers;
+//   warp 1      allocates tensor memory, one lane issues tcgen05.mma (128 x BN x 16, f32
+//               accumulation in TMEM) and commits stage releases / accumulator readiness;
+//   warps 2..5  read the accumulator with tcgen05.ld (one row per thread) and apply the fused
+//               epilogue while the MMA warp already fills the other accumulator buffer.
+// Every mbarrier wait is bounded; on a timeout the CTA sets an error word, drains its own
+// TMA copies, frees its tensor memory and returns.
+#include "wf_internal.h"
+#include "wf_epilogue.cuh"
+#include "wf_ptx.cuh"
+
+namespace wf {
+
+using namespace ptx;
+
+constexpr int kBM = 128;
+constexpr int kBK = 64;
+constexpr int kGemmThreads = 192;
+
+template <int BN>
+struct GemmCfg {
+  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static constexpr int kABytes = kBM * kBK * 2;
+  static constexpr int kBBytes = BN * kBK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kBarOffset = kStages * kStageBytes;
+  static constexpr int kSmemBytes = kBarOffset + 256 + 1024;  // barriers + alignment slack
+  static constexpr int kTmemCols = 2 * BN;
+};
+
+// One accumulator row segment: 32 consecutive columns starting at col0 for GEMM row `row`.
+template <int EPI>
+__device__ __forceinline__ void epilogue_row32(const EpiParams& ep, long row, long M, int col0, int N,
+                                               const uint32_t (&acc)[32]) {
+  if (row >= M || col0 >= N) return;
+  long orow = row;
+  bool valid = true;
+  int pos = 0;
+  if (EPI == kEpiConv1) valid = ep.row_valid[row] != 0;
+  if (EPI == kEpiConv2) {
+    int2 d = ep.row_dst[row];
+    if (d.x < 0) return;
+    orow = d.x;
+    pos = d.y;
+  }
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {  // groups of 8 columns
+    int col = col0 + 8 * g;
+    if (col >= N) break;
+    float v[8];
+    float4 b0 = __ldg(reinterpret_cast<const float4*>(ep.bias + col));
+    float4 b1 = __ldg(reinterpret_cast<const float4*>(ep.bias + col + 4));
+    v[0] = __uint_as_float(acc[8 * g + 0]) + b0.x;
+    v[1] = __uint_as_float(acc[8 * g + 1]) + b0.y;
+    v[2] = __uint_as_float(acc[8 * g + 2]) + b0.z;
+    v[3] = __uint_as_float(acc[8 * g + 3]) + b0.w;
+    v[4] = __uint_as_float(acc[8 * g + 4]) + b1.x;
+    v[5] = __uint_as_float(acc[8 * g + 5]) + b1.y;
+    v[6] = __uint_as_float(acc[8 * g + 6]) + b1.z;
+    v[7] = __uint_as_float(acc[8 * g + 7]) + b1.w;
+    if (EPI == kEpiBiasGelu || EPI == kEpiConv1 || EPI == kEpiConv2) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = gelu_erf(v[i]);
+    }
+    if (EPI == kEpiBias || EPI == kEpiBiasGelu || EPI == kEpiConv1) {
+      if (EPI == kEpiConv1 && !valid) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = 0.f;
+      }
+      __nv_bfloat162 p0 = __floats2bfloat162_rn(v[0], v[1]), p1 = __floats2bfloat162_rn(v[2], v[3]);
+      __nv_bfloat162 p2 = __floats2bfloat162_rn(v[4], v[5]), p3 = __floats2bfloat162_rn(v[6], v[7]);
+      uint4 u;
+      u.x = *reinterpret_cast<uint32_t*>(&p0);
+      u.y = *reinterpret_cast<uint32_t*>(&p1);
+      u.z = *reinterpret_cast<uint32_t*>(&p2);
+      u.w = *reinterpret_cast<uint32_t*>(&p3);
+      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.out) + orow * ep.ldc + col) = u;
+    } else if (EPI == kEpiBiasResid) {
+      float4* p = reinterpret_cast<float4*>(ep.resid + orow * ep.ldc + col);
+      float4 r0 = p[0], r1 = p[1];
+      r0.x += v[0]; r0.y += v[1]; r0.z += v[2]; r0.w += v[3];
+      r1.x += v[4]; r1.y += v[5]; r1.z += v[6]; r1.w += v[7];
+      p[0] = r0;
+      p[1] = r1;
+    } else {  // kEpiConv2
+      const float4* pe = reinterpret_cast<const float4*>(ep.pe + (long)pos * ep.ldc + col);
+      float4 e0 = __ldg(pe), e1 = __ldg(pe + 1);
+      float4* p = reinterpret_cast<float4*>(ep.resid + orow * ep.ldc + col);
+      p[0] = make_float4(v[0] + e0.x, v[1] + e0.y, v[2] + e0.z, v[3] + e0.w);
+      p[1] = make_float4(v[4] + e1.x, v[5] + e1.y, v[6] + e1.z, v[7] + e1.w);
+    }
+  }
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
+    const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, long M, int N,
+    int K, int a_cols, EpiParams ep, int* err_flag) {
+  using Cfg = GemmCfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + Cfg::kBarOffset;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (Cfg::kStages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * Cfg::kStages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * Cfg::kStages + 2 + a); };
+  volatile uint32_t* tmem_slot =
+      reinterpret_cast<volatile uint32_t*>(smem_gen + Cfg::kBarOffset + 8 * (2 * Cfg::kStages + 4));
+  volatile int* abort_flag =
+      reinterpret_cast<volatile int*>(smem_gen + Cfg::kBarOffset + 8 * (2 * Cfg::kStages + 4) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 4);
+    }
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int num_m = (int)((M + kBM - 1) / kBM);
+  const int num_n = (N + BN - 1) / BN;
+  const int num_k = (K + kBK - 1) / kBK;
+  const int num_tiles = num_m * num_n;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&tmap_a);
+      prefetch_tmap(&tmap_b);
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t armed = 0, armed_parity = 0;  // bit s: stage s has had a load issued / its parity
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        const int m0 = (tile / num_n) * kBM, n0 = (tile % num_n) * BN;
+        for (int kb = 0; kb < num_k; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageBytes);
+          const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
+          // A row of the GEMM may wrap over consecutive rows of the stored matrix (conv stem:
+          // three time rows laid end to end); a_cols is the stored row length, K for a plain GEMM.
+          const int e = kb * kBK;
+          tma_load_2d(sa, &tmap_a, e % a_cols, m0 + e / a_cols, full_bar(stage));
+          tma_load_2d(sa + Cfg::kABytes, &tmap_b, kb * kBK, n0, full_bar(stage));
+          armed |= 1u << stage;
+          armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+          if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        atomicExch(err_flag, 1);
+        // Let the copies this thread issued land before the CTA's shared memory is released.
+        for (int s = 0; s < Cfg::kStages; ++s) {
+          if (!(armed & (1u << s))) continue;
+          for (uint32_t it = 0; it < (1u << 20); ++it)
+            if (mbar_try_wait(full_bar(s), (armed_parity >> s) & 1u)) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN, 0, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_k; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
+          const uint64_t adesc = umma_desc_k_sw128(sa);
+          const uint64_t bdesc = umma_desc_k_sw128(sa + Cfg::kABytes);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) {
+            // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte units
+            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));
+          if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(tfull_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (!ok) atomicExch(err_flag, 2);
+    }
+  } else {
+    const int quarter = warp & 3;  // TMEM lanes this warp may read: 32 * quarter .. + 31
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+      const int m0 = (tile / num_n) * kBM, n0 = (tile % num_n) * BN;
+      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) {
+        if (lane == 0) atomicExch(err_flag, 3);
+        break;
+      }
+      tc_fence_after();
+      const long row = (long)m0 + quarter * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld_32x32(t_row + c * 32, v);
+        tmem_ld_wait();
+        epilogue_row32<EPI>(ep, row, M, n0 + c * 32, N, v);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+bool tma_api_init(TmaApi* api) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || fn == nullptr) return false;
+  api->encode_tiled = fn;
+  return true;
+}
+
+bool make_tmap_bf16(const TmaApi& api, CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows,
+                    uint64_t pitch_elems, uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {pitch_elems * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = reinterpret_cast<EncodeTiledFn>(api.encode_tiled)(
+      m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <int BN, int EPI>
+static cudaError_t configure_one() {
+  return cudaFuncSetAttribute(gemm_bf16_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              GemmCfg<BN>::kSmemBytes);
+}
+
+cudaError_t gemm_bf16_configure() {
+  cudaError_t e;
+  if ((e = configure_one<256, kEpiBias>()) != cudaSuccess) return e;
+  if ((e = configure_one<256, kEpiBiasGelu>()) != cudaSuccess) return e;
+  if ((e = configure_one<256, kEpiBiasResid>()) != cudaSuccess) return e;
+  if ((e = configure_one<256, kEpiConv1>()) != cudaSuccess) return e;
+  if ((e = configure_one<256, kEpiConv2>()) != cudaSuccess) return e;
+  return cudaSuccess;
+}
+
+template <int BN, int EPI>
+static void launch_one(const CUtensorMap& ta, const CUtensorMap& tb, long M, int N, int K, int a_cols,
+                       const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
+  const long tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
+  const int grid = (int)(tiles < num_sms ? tiles : num_sms);
+  gemm_bf16_kernel<BN, EPI><<<grid, kGemmThreads, GemmCfg<BN>::kSmemBytes, s>>>(ta, tb, M, N, K, a_cols, ep,
+                                                                                 err_flag);
+}
+
+void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, long M, int N, int K, int a_cols,
+                      int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
+  if (M <= 0 || N <= 0 || K <= 0) return;
+  switch (epi) {
+    case kEpiBias: launch_one<256, kEpiBias>(ta, tb, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    case kEpiBiasGelu: launch_one<256, kEpiBiasGelu>(ta, tb, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    case kEpiBiasResid: launch_one<256, kEpiBiasResid>(ta, tb, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    case kEpiConv1: launch_one<256, kEpiConv1>(ta, tb, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    default: launch_one<256, kEpiConv2>(ta, tb, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+  }
+}
+
+}  // namespace wf

@@ -1,0 +1,101 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/wf_encoder.h"
+
+namespace wf {
+
+constexpr int kNFft = 400;
+constexpr int kHop = 160;
+constexpr int kBins = 201;
+constexpr int kFold = 200;        // folded DFT length: 400-point real input, symmetric window
+constexpr int kBasisCols = 224;   // 201 bins padded to 7 x 32 lanes
+constexpr int kFeFrames = 64;     // frames per front-end CTA
+constexpr int kHeadDim = 64;
+
+// Epilogue selectors shared by the SIMT and the tcgen05 GEMM kernels.
+enum Epilogue : int {
+  kEpiBias = 0,       // out = acc + bias
+  kEpiBiasGelu = 1,   // out = gelu(acc + bias)
+  kEpiBiasResid = 2,  // resid(f32) += acc + bias
+  kEpiConv1 = 3,      // out[row] = row_valid[row] ? gelu(acc + bias) : 0
+  kEpiConv2 = 4       // resid(f32)[dst[row]] = gelu(acc + bias) + pe[pos[row]] (dst < 0: skip)
+};
+
+struct EpiParams {
+  const float* bias;     // [N]
+  void* out;             // element type of the path (kEpiBias, kEpiBiasGelu, kEpiConv1)
+  float* resid;          // f32 (kEpiBiasResid, kEpiConv2)
+  long ldc;              // leading dimension of out / resid (and of pe) in elements
+  const int* row_valid;  // kEpiConv1: one int per GEMM row
+  const int2* row_dst;   // kEpiConv2: (destination token row or -1, position in sequence)
+  const float* pe;       // kEpiConv2: sinusoid table [n_ctx, N]
+};
+
+// Offsets (in ints) of the per-call metadata arrays inside one device int buffer.
+struct MetaLayout {
+  int sample_off;   // [B+1] first sample of each buffer in the packed audio
+  int frames;       // [B]   audio frames T_i
+  int frame_off;    // [B+1] prefix sums of T_i
+  int prow_off;     // [B+1] first row of each sequence in the padded-row layout (even)
+  int tok_off;      // [B+1] token prefix sums (cu_seqlens)
+  int fe_tile_off;  // [B+1] prefix sums of front-end tiles
+  int attn_work;    // [n_attn_work] pairs (sequence, first query row within the sequence)
+  int total;
+};
+
+// ---- tables (wf_frontend.cu)
+void launch_build_tables(float* dft_basis /*[2][kFold][kBasisCols]*/, float* pe, int n_ctx, int d,
+                         cudaStream_t s);
+
+// ---- front end (wf_frontend.cu)
+void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, int n_tiles,
+                     const float* dft_basis, const float* mel_fb_t /*[201][n_mel]*/, int n_mel,
+                     float* logmel /*[sum T, n_mel]*/, int* seq_max /*[B] ordered ints*/,
+                     cudaStream_t s);
+// mode 0: packed normalised mel (float) for wf_logmel; mode 1: padded-row layout + hush rows.
+void launch_normalise(const float* logmel, const int* seq_max, const float* mel_in,
+                      const int* meta, MetaLayout ml, int B, int max_rows, int n_mel, int dst_ld,
+                      int hush_frames, const float* hush, void* dst, int dst_bf16, int mode, cudaStream_t s);
+void launch_build_maps(const int* meta, MetaLayout ml, int B, int max_rows, int hush_frames,
+                       int* row_valid, int2* row_dst, cudaStream_t s);
+void launch_fill_seq_max(int* seq_max, int B, cudaStream_t s);
+
+// ---- SIMT float32 kernels and element-wise kernels (wf_simt.cu)
+void launch_gemm_f32(const float* A, long lda, const float* W, long ldw, long M, int N, int K,
+                     int epi, const EpiParams& ep, cudaStream_t s);
+void launch_layernorm(const float* x, const float* g, const float* b, void* out, int out_bf16,
+                      long M, int d, cudaStream_t s);
+void launch_attention_f32(const float* qkv, float* out, const int* meta, MetaLayout ml, int n_work,
+                          int d_model, cudaStream_t s);
+void launch_convert(const float* src, void* dst, long n, int dst_bf16, cudaStream_t s);
+void launch_conv_weight(const float* src /*[out, in, 3]*/, void* dst /*[out, 3*in_ld], zeroed*/, int c_out,
+                        int c_in, int in_ld, int dst_bf16, cudaStream_t s);
+void launch_transpose_f32(const float* src, float* dst, int rows, int cols, cudaStream_t s);
+
+// ---- tcgen05 bf16 GEMM (wf_gemm_tcgen05.cu)
+struct TmaApi {
+  void* encode_tiled;  // cuTensorMapEncodeTiled
+};
+bool tma_api_init(TmaApi* api);
+// 2-D bf16 tensor map: inner extent `cols` (elements), outer extent `rows`, row pitch in
+// elements, box = 64 x box_rows, 128 B swizzle.
+bool make_tmap_bf16(const TmaApi& api, CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows,
+                    uint64_t pitch_elems, uint32_t box_rows);
+cudaError_t gemm_bf16_configure();
+// a_cols: stored row length of A in elements (K for a plain GEMM; smaller when one GEMM row
+// spans several consecutive stored rows, which must then be a multiple of 64).
+void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, long M, int N, int K, int a_cols,
+                      int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s);
+
+// ---- bf16 attention (wf_attention.cu)
+cudaError_t attention_bf16_configure();
+void launch_attention_bf16(const __nv_bfloat16* qkv, __nv_bfloat16* out, const int* meta,
+                           MetaLayout ml, int n_work, int d_model, cudaStream_t s);
+
+}  // namespace wf
