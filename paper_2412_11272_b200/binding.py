@@ -1,0 +1,250 @@
+"""ctypes binding of libwf_encoder.so: argument marshalling only.
+
+Every step of the encoding path runs inside the library's CUDA kernels; this module turns
+torch tensors into pointers, keeps them alive, and raises on error codes.  PyTorch is used
+for device memory and streams, nothing else.  There is no CPU fallback: if the shared
+library is missing or cannot be loaded, importing the handle raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libwf_encoder.so")
+
+WF_F32, WF_BF16 = 0, 1
+STATUS = {0: "WF_OK", 1: "WF_ERR_INVALID_ARG", 2: "WF_ERR_TOO_SHORT", 3: "WF_ERR_TOO_LONG",
+          4: "WF_ERR_CAPACITY", 5: "WF_ERR_CUDA", 6: "WF_ERR_DEVICE_TIMEOUT",
+          7: "WF_ERR_UNSUPPORTED_ARCH", 8: "WF_ERR_UNIMPLEMENTED"}
+N_KERNEL_CLASSES = 6
+KERNEL_CLASSES = ("front_end", "layout", "conv_gemm", "layernorm", "block_gemm", "attention")
+
+
+class WfError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"{STATUS.get(code, code)}: {message}")
+        self.code = code
+        self.status = STATUS.get(code, str(code))
+
+
+class wf_config(C.Structure):
+    _fields_ = [("n_mel", C.c_int), ("d_model", C.c_int), ("n_layer", C.c_int), ("n_head", C.c_int),
+                ("d_mlp", C.c_int), ("n_ctx", C.c_int), ("hush_frames", C.c_int), ("dtype", C.c_int),
+                ("max_batch", C.c_int), ("max_tokens", C.c_long), ("max_samples", C.c_long)]
+
+
+_PP = C.POINTER(C.c_void_p)
+
+
+class wf_weights(C.Structure):
+    _fields_ = [("mel_fb", C.c_void_p), ("conv1_w", C.c_void_p), ("conv1_b", C.c_void_p),
+                ("conv2_w", C.c_void_p), ("conv2_b", C.c_void_p),
+                ("ln1_g", _PP), ("ln1_b", _PP), ("wq", _PP), ("bq", _PP), ("wk", _PP), ("wv", _PP),
+                ("bv", _PP), ("wo", _PP), ("bo", _PP), ("ln2_g", _PP), ("ln2_b", _PP),
+                ("w1", _PP), ("b1", _PP), ("w2", _PP), ("b2", _PP),
+                ("lnp_g", C.c_void_p), ("lnp_b", C.c_void_p)]
+
+
+_PER_LAYER = ("ln1_g", "ln1_b", "wq", "bq", "wk", "wv", "bv", "wo", "bo", "ln2_g", "ln2_b",
+              "w1", "b1", "w2", "b2")
+
+EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_mel", "wf_encode_host", "wf_check",
+           "wf_encoder_destroy", "wf_last_error", "wf_profile_enable", "wf_profile_read",
+           "wf_gemm_bf16", "wf_attention")
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads the shared library (building it is the job of ``paper_2412_11272_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(f"{LIB_PATH} is missing: run `python -m paper_2412_11272_b200.build`")
+    lib = C.CDLL(LIB_PATH)
+    vp, ip, lp = C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_long)
+    lib.wf_encoder_create.argtypes = [C.POINTER(wf_config), C.POINTER(wf_weights), vp, C.POINTER(vp)]
+    lib.wf_logmel.argtypes = [vp, vp, lp, C.c_int, vp, lp, vp]
+    lib.wf_encode.argtypes = [vp, vp, lp, C.c_int, vp, vp, ip, vp]
+    lib.wf_encode_mel.argtypes = [vp, vp, lp, C.c_int, vp, vp, ip, vp]
+    lib.wf_encode_host.argtypes = [vp, vp, lp, C.c_int, vp, vp, ip, vp]
+    lib.wf_check.argtypes = [vp, vp]
+    lib.wf_encoder_destroy.argtypes = [vp]
+    lib.wf_last_error.argtypes = [vp]
+    lib.wf_last_error.restype = C.c_char_p
+    lib.wf_profile_enable.argtypes = [vp, C.c_int]
+    lib.wf_profile_read.argtypes = [vp, lp, C.POINTER(C.c_double)]
+    lib.wf_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, C.c_long, C.c_int, C.c_int, C.c_int, vp]
+    lib.wf_attention.argtypes = [vp, vp, ip, C.c_int, vp, vp]
+    for name in EXPORTS:
+        if name != "wf_last_error":
+            getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _stream_ptr(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _longs(values):
+    arr = np.ascontiguousarray(np.asarray(values, dtype=np.int64))
+    return arr, arr.ctypes.data_as(C.POINTER(C.c_long))
+
+
+class Encoder:
+    """Owns one ``wf_encoder`` handle.  ``weights`` maps the names of
+    ``inputs.encoder_weights`` to float32 arrays (numpy or torch); they are moved to the
+    current CUDA device and may be released by the caller afterwards."""
+
+    def __init__(self, shape, weights: dict, mel_fb, max_batch: int, max_tokens: int, max_samples: int,
+                 hush_frames: int | None = None, n_ctx: int | None = None, dtype: str | None = None,
+                 device="cuda:0"):
+        self.lib = load_library()
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.shape = shape
+        self.dtype = dtype or shape.dtype
+        self.hush_frames = shape.hush_frames if hush_frames is None else hush_frames
+        self.n_ctx = shape.n_ctx if n_ctx is None else n_ctx
+        self.d_model = shape.d_model
+        self.n_mel = shape.n_mel
+        self.out_dtype = torch.bfloat16 if self.dtype == "bf16" else torch.float32
+        cfg = wf_config(shape.n_mel, shape.d_model, shape.n_layer, shape.n_head, shape.d_mlp, self.n_ctx,
+                        self.hush_frames, WF_BF16 if self.dtype == "bf16" else WF_F32,
+                        int(max_batch), int(max_tokens), int(max_samples))
+        dev = {}
+
+        def put(a):
+            t = torch.as_tensor(np.ascontiguousarray(a) if isinstance(a, np.ndarray) else a)
+            return t.to(device=self.device, dtype=torch.float32).contiguous()
+
+        w = wf_weights()
+        for name in ("conv1_w", "conv1_b", "conv2_w", "conv2_b", "lnp_g", "lnp_b"):
+            dev[name] = put(weights[name])
+            setattr(w, name, dev[name].data_ptr())
+        dev["mel_fb"] = put(mel_fb)
+        w.mel_fb = dev["mel_fb"].data_ptr()
+        arrays = {}
+        for name in _PER_LAYER:
+            arr = (C.c_void_p * max(shape.n_layer, 1))()
+            for l in range(shape.n_layer):
+                dev[f"{name}.{l}"] = put(weights[f"{name}.{l}"])
+                arr[l] = dev[f"{name}.{l}"].data_ptr()
+            arrays[name] = arr
+            setattr(w, name, C.cast(arr, _PP))
+        handle = C.c_void_p()
+        st = self.lib.wf_encoder_create(C.byref(cfg), C.byref(w), _stream_ptr(), C.byref(handle))
+        self.handle = handle
+        if st != 0:
+            msg = self.lib.wf_last_error(handle).decode() if handle else "create failed"
+            if handle:
+                self.lib.wf_encoder_destroy(handle)
+            self.handle = None
+            raise WfError(st, msg)
+        torch.cuda.synchronize()
+        del dev, arrays  # the library holds its own converted copies
+
+    # -- helpers
+    def _check(self, st: int):
+        if st != 0:
+            raise WfError(st, self.lib.wf_last_error(self.handle).decode())
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.wf_encoder_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- entry points (same names as the C ABI)
+    def wf_logmel(self, audio: torch.Tensor, lengths, stream=None):
+        """audio: float32 CUDA tensor of packed samples.  Returns (mel [sum T, n_mel] f32, frames)."""
+        arr, ptr = _longs(lengths)
+        B = len(arr)
+        total_frames = int((arr // 160).sum())
+        mel = torch.empty((total_frames, self.n_mel), dtype=torch.float32, device=self.device)
+        frames = np.zeros(max(B, 1), dtype=np.int64)
+        self._check(self.lib.wf_logmel(self.handle, audio.data_ptr() if B else None, ptr, B, mel.data_ptr(),
+                                       frames.ctypes.data_as(C.POINTER(C.c_long)), _stream_ptr(stream)))
+        return mel, frames[:B]
+
+    def _tokens(self, frames):
+        return (np.asarray(frames, dtype=np.int64) + self.hush_frames + 1) // 2
+
+    def wf_encode(self, audio: torch.Tensor, lengths, hush_mel: torch.Tensor | None, out=None, stream=None):
+        """Returns (hidden [sum n_i, d_model], cu_seqlens int32 numpy [B+1]).  No host sync."""
+        arr, ptr = _longs(lengths)
+        B = len(arr)
+        M = int(self._tokens(arr // 160).sum())
+        if out is None:
+            out = torch.empty((M, self.d_model), dtype=self.out_dtype, device=self.device)
+        cu = np.zeros(B + 1, dtype=np.int32)
+        self._check(self.lib.wf_encode(self.handle, audio.data_ptr() if B else None, ptr, B,
+                                       hush_mel.data_ptr() if hush_mel is not None else None,
+                                       out.data_ptr(), cu.ctypes.data_as(C.POINTER(C.c_int)),
+                                       _stream_ptr(stream)))
+        return out, cu
+
+    def wf_encode_mel(self, mel: torch.Tensor, frames, hush_mel, out=None, stream=None):
+        arr, ptr = _longs(frames)
+        B = len(arr)
+        M = int(self._tokens(arr).sum())
+        if out is None:
+            out = torch.empty((M, self.d_model), dtype=self.out_dtype, device=self.device)
+        cu = np.zeros(B + 1, dtype=np.int32)
+        self._check(self.lib.wf_encode_mel(self.handle, mel.data_ptr() if B else None, ptr, B,
+                                           hush_mel.data_ptr() if hush_mel is not None else None,
+                                           out.data_ptr(), cu.ctypes.data_as(C.POINTER(C.c_int)),
+                                           _stream_ptr(stream)))
+        return out, cu
+
+    def wf_encode_host(self, audio_host: torch.Tensor, lengths, hush_mel, out_host: torch.Tensor, stream=None):
+        """audio_host / out_host: (pinned) CPU tensors.  Copies in, encodes, copies out, synchronises."""
+        arr, ptr = _longs(lengths)
+        B = len(arr)
+        cu = np.zeros(B + 1, dtype=np.int32)
+        self._check(self.lib.wf_encode_host(self.handle, audio_host.data_ptr(), ptr, B,
+                                            hush_mel.data_ptr() if hush_mel is not None else None,
+                                            out_host.data_ptr(), cu.ctypes.data_as(C.POINTER(C.c_int)),
+                                            _stream_ptr(stream)))
+        return out_host, cu
+
+    def wf_check(self, stream=None):
+        self._check(self.lib.wf_check(self.handle, _stream_ptr(stream)))
+
+    def wf_profile_enable(self, on: bool):
+        self._check(self.lib.wf_profile_enable(self.handle, 1 if on else 0))
+
+    def wf_profile_read(self) -> dict:
+        n = (C.c_long * N_KERNEL_CLASSES)()
+        ms = (C.c_double * N_KERNEL_CLASSES)()
+        self._check(self.lib.wf_profile_read(self.handle, n, ms))
+        return {KERNEL_CLASSES[i]: {"launches": int(n[i]), "ms": float(ms[i])} for i in range(N_KERNEL_CLASSES)}
+
+    def wf_gemm_bf16(self, A: torch.Tensor, W: torch.Tensor, bias: torch.Tensor, mode: int, C_out=None,
+                     stream=None):
+        M, K = A.shape
+        N = W.shape[0]
+        if C_out is None:
+            C_out = torch.empty((M, N), dtype=torch.bfloat16, device=A.device)
+        self._check(self.lib.wf_gemm_bf16(self.handle, A.data_ptr(), W.data_ptr(), bias.data_ptr(),
+                                          C_out.data_ptr(), M, N, K, mode, _stream_ptr(stream)))
+        return C_out
+
+    def wf_attention(self, qkv: torch.Tensor, cu_seqlens, stream=None):
+        cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+        out = torch.empty((qkv.shape[0], self.d_model), dtype=qkv.dtype, device=qkv.device)
+        self._check(self.lib.wf_attention(self.handle, qkv.data_ptr(), cu.ctypes.data_as(C.POINTER(C.c_int)),
+                                          len(cu) - 1, out.data_ptr(), _stream_ptr(stream)))
+        return out

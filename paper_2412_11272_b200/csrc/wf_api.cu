@@ -1,0 +1,700 @@
+// C ABI, host-side ragged planner and launch sequence of the encoder.
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "wf_internal.h"
+
+using namespace wf;
+
+namespace {
+constexpr int kRing = 4;          // per-call metadata slots (pinned host + device)
+constexpr int kMinSamples = 401;  // reflect padding of 200 needs more than 200 samples on each side
+}  // namespace
+
+struct LayerW {
+  float *ln1_g, *ln1_b, *ln2_g, *ln2_b;
+  void *wqkv, *wo, *w1, *w2;
+  float *bqkv, *bo, *b1, *b2;
+  CUtensorMap tm_wqkv, tm_wo, tm_w1, tm_w2;
+};
+
+struct ProfEvent {
+  cudaEvent_t a, b;
+  int cls;
+};
+
+struct wf_encoder {
+  wf_config cfg;
+  bool bf16;
+  int num_sms;
+  size_t esz;
+  int mel_ld;      // channels per stored log-mel row (n_mel, rounded up to 64 on the bf16 path)
+  long cap_prows;  // padded-row capacity
+  char err[512];
+  std::vector<void*> allocs;
+  std::vector<void*> pinned;
+  TmaApi tma;
+
+  float *dft_basis, *pe, *mel_fb_t;
+  void *conv1_w, *conv2_w;
+  float *conv1_b, *conv2_b, *lnp_g, *lnp_b;
+  std::vector<LayerW> layers;
+  CUtensorMap tm_conv1_w, tm_conv2_w, tm_zp, tm_c1p, tm_h, tm_attn, tm_fc1;
+
+  float* logmel;
+  int* seq_max;
+  void *zp_alloc, *c1p;
+  int* row_valid;
+  int2* row_dst;
+  float* x;
+  void *h, *qkv, *attn, *fc1;
+  float* audio_stage;
+  void* out_stage;
+  int* err_flag;
+
+  int meta_cap;
+  int* meta_dev[kRing];
+  int* meta_host[kRing];
+  cudaEvent_t meta_ev[kRing];
+  bool meta_used[kRing];
+  int ring_pos;
+
+  bool profile;
+  std::vector<ProfEvent> prof;
+  size_t prof_used;
+};
+
+namespace {
+
+struct Plan {
+  int B;
+  long total_samples;
+  int total_frames, total_prows, total_tokens;
+  int n_fe_tiles, n_work, max_prows_seq;
+  MetaLayout ml;
+};
+
+wf_status fail(wf_encoder* e, wf_status st, const char* fmt, ...) {
+  if (e) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(e->err, sizeof(e->err), fmt, ap);
+    va_end(ap);
+  }
+  return st;
+}
+
+#define WF_CUDA(e, call)                                                                     \
+  do {                                                                                       \
+    cudaError_t _c = (call);                                                                 \
+    if (_c != cudaSuccess)                                                                   \
+      return fail((e), WF_ERR_CUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(_c),  \
+                  __FILE__, __LINE__);                                                       \
+  } while (0)
+
+template <typename T>
+wf_status dev_alloc(wf_encoder* e, T** p, size_t n_elems, bool zero = false) {
+  void* q = nullptr;
+  size_t bytes = std::max<size_t>(n_elems * sizeof(T), 256);
+  WF_CUDA(e, cudaMalloc(&q, bytes));
+  e->allocs.push_back(q);
+  if (zero) WF_CUDA(e, cudaMemset(q, 0, bytes));
+  *p = reinterpret_cast<T*>(q);
+  return WF_OK;
+}
+
+wf_status dev_alloc_bytes(wf_encoder* e, void** p, size_t bytes, bool zero = false) {
+  uint8_t* q = nullptr;
+  wf_status st = dev_alloc<uint8_t>(e, &q, bytes, zero);
+  *p = q;
+  return st;
+}
+
+// Copies a float32 device vector into library-owned memory.
+wf_status own_f32(wf_encoder* e, float** dst, const float* src, size_t n, cudaStream_t s) {
+  if (!src) return fail(e, WF_ERR_INVALID_ARG, "a weight pointer is NULL");
+  wf_status st = dev_alloc<float>(e, dst, n);
+  if (st != WF_OK) return st;
+  WF_CUDA(e, cudaMemcpyAsync(*dst, src, n * sizeof(float), cudaMemcpyDeviceToDevice, s));
+  return WF_OK;
+}
+
+// Converts a float32 device matrix into the path's element type at dst (+ element offset).
+wf_status own_mat(wf_encoder* e, void* dst, size_t elem_off, const float* src, size_t n, cudaStream_t s) {
+  if (!src) return fail(e, WF_ERR_INVALID_ARG, "a weight pointer is NULL");
+  launch_convert(src, (uint8_t*)dst + elem_off * e->esz, (long)n, e->bf16 ? 1 : 0, s);
+  return WF_OK;
+}
+
+class Prof {
+ public:
+  Prof(wf_encoder* e, int cls, cudaStream_t s) : e_(e), s_(s), ev_(nullptr) {
+    if (!e->profile) return;
+    if (e->prof_used == e->prof.size()) {
+      ProfEvent pe;
+      if (cudaEventCreate(&pe.a) != cudaSuccess || cudaEventCreate(&pe.b) != cudaSuccess) return;
+      pe.cls = cls;
+      e->prof.push_back(pe);
+    }
+    ev_ = &e->prof[e->prof_used++];
+    ev_->cls = cls;
+    cudaEventRecord(ev_->a, s_);
+  }
+  ~Prof() {
+    if (ev_) cudaEventRecord(ev_->b, s_);
+  }
+
+ private:
+  wf_encoder* e_;
+  cudaStream_t s_;
+  ProfEvent* ev_;
+};
+
+// Builds prefix sums, the padded-row layout and the work lists for one call into `hm`
+// (host ints), validating every length.  `frames_given`: `len` holds frame counts, not samples.
+wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Plan* p, int* hm,
+                    bool build_work = true) {
+  const wf_config& c = e->cfg;
+  if (B < 0 || (B > 0 && !len)) return fail(e, WF_ERR_INVALID_ARG, "bad batch size or NULL lengths");
+  if (B > c.max_batch) return fail(e, WF_ERR_CAPACITY, "batch %d exceeds max_batch %d", B, c.max_batch);
+  MetaLayout& ml = p->ml;
+  int off = 0;
+  ml.sample_off = off; off += B + 1;
+  ml.frames = off; off += B + 1;
+  ml.frame_off = off; off += B + 1;
+  ml.prow_off = off; off += B + 1;
+  ml.tok_off = off; off += B + 1;
+  ml.fe_tile_off = off; off += B + 1;
+  ml.attn_work = off;
+  long samples = 0, frames = 0, prows = 0, tokens = 0, tiles = 0;
+  int max_pr = 0;
+  for (int i = 0; i < B; ++i) {
+    long L = len[i], T;
+    if (frames_given) {
+      if (L < 1) return fail(e, WF_ERR_TOO_SHORT, "sequence %d has %ld frames", i, L);
+      T = L;
+      L = 0;
+    } else {
+      if (L < kMinSamples) return fail(e, WF_ERR_TOO_SHORT, "buffer %d has %ld samples (need >= %d)", i, L, kMinSamples);
+      T = L / kHop;
+    }
+    long rows = T + c.hush_frames;
+    long n = (rows + 1) / 2;
+    if (n > c.n_ctx) return fail(e, WF_ERR_TOO_LONG, "sequence %d would have %ld tokens (n_ctx %d)", i, n, c.n_ctx);
+    hm[ml.sample_off + i] = (int)samples;
+    hm[ml.frames + i] = (int)T;
+    hm[ml.frame_off + i] = (int)frames;
+    hm[ml.prow_off + i] = (int)prows;
+    hm[ml.tok_off + i] = (int)tokens;
+    hm[ml.fe_tile_off + i] = (int)tiles;
+    samples += L;
+    frames += T;
+    prows += 2 * (n + 1);
+    tokens += n;
+    tiles += (T + kFeFrames - 1) / kFeFrames;
+    max_pr = std::max<int>(max_pr, (int)(2 * (n + 1)));
+    if (samples > c.max_samples) return fail(e, WF_ERR_CAPACITY, "more than max_samples=%ld samples", c.max_samples);
+    if (tokens > c.max_tokens) return fail(e, WF_ERR_CAPACITY, "more than max_tokens=%ld tokens", c.max_tokens);
+  }
+  hm[ml.sample_off + B] = (int)samples;
+  hm[ml.frames + B] = 0;
+  hm[ml.frame_off + B] = (int)frames;
+  hm[ml.prow_off + B] = (int)prows;
+  hm[ml.tok_off + B] = (int)tokens;
+  hm[ml.fe_tile_off + B] = (int)tiles;
+  // attention work list: (sequence, first query row), longest sequences first
+  const int qt = e->bf16 ? 64 : 16;
+  std::vector<int> order(B);
+  for (int i = 0; i < B; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+    return hm[ml.tok_off + a + 1] - hm[ml.tok_off + a] > hm[ml.tok_off + b + 1] - hm[ml.tok_off + b];
+  });
+  int nw = 0;
+  for (int oi = 0; build_work && oi < B; ++oi) {
+    int i = order[oi];
+    int n = hm[ml.tok_off + i + 1] - hm[ml.tok_off + i];
+    for (int q0 = 0; q0 < n; q0 += qt) {
+      hm[ml.attn_work + 2 * nw] = i;
+      hm[ml.attn_work + 2 * nw + 1] = q0;
+      ++nw;
+    }
+  }
+  ml.total = ml.attn_work + 2 * nw;
+  p->B = B;
+  p->total_samples = samples;
+  p->total_frames = (int)frames;
+  p->total_prows = (int)prows;
+  p->total_tokens = (int)tokens;
+  p->n_fe_tiles = (int)tiles;
+  p->n_work = nw;
+  p->max_prows_seq = max_pr;
+  return WF_OK;
+}
+
+wf_status ring_acquire(wf_encoder* e, int* slot) {
+  int s = e->ring_pos;
+  e->ring_pos = (e->ring_pos + 1) % kRing;
+  if (e->meta_used[s]) WF_CUDA(e, cudaEventSynchronize(e->meta_ev[s]));
+  *slot = s;
+  return WF_OK;
+}
+
+wf_status ring_upload(wf_encoder* e, int slot, const Plan& p, cudaStream_t s) {
+  WF_CUDA(e, cudaMemcpyAsync(e->meta_dev[slot], e->meta_host[slot], (size_t)std::max(p.ml.total, 1) * sizeof(int),
+                             cudaMemcpyHostToDevice, s));
+  return WF_OK;
+}
+
+wf_status ring_release(wf_encoder* e, int slot, cudaStream_t s) {
+  WF_CUDA(e, cudaEventRecord(e->meta_ev[slot], s));
+  e->meta_used[slot] = true;
+  return WF_OK;
+}
+
+void gemm(wf_encoder* e, const CUtensorMap* ta, const CUtensorMap* tb, const void* A, long lda, const void* W,
+          long ldw, long M, int N, int K, int a_cols, int epi, const EpiParams& ep, cudaStream_t s) {
+  if (e->bf16) launch_gemm_bf16(*ta, *tb, M, N, K, a_cols, epi, ep, e->err_flag, e->num_sms, s);
+  else launch_gemm_f32((const float*)A, lda, (const float*)W, ldw, M, N, K, epi, ep, s);
+}
+
+// Everything after the log-mel rows sit in the padded-row layout.
+wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidden_out, cudaStream_t s) {
+  const wf_config& c = e->cfg;
+  const int d = c.d_model, F = c.d_mlp;
+  const long M = p.total_tokens;
+  const int bf = e->bf16 ? 1 : 0;
+  {
+    Prof pr(e, 1, s);
+    launch_build_maps(meta, p.ml, p.B, p.max_prows_seq, c.hush_frames, e->row_valid, e->row_dst, s);
+  }
+  {
+    Prof pr(e, 2, s);
+    EpiParams ep{};
+    ep.bias = e->conv1_b; ep.out = e->c1p; ep.ldc = d; ep.row_valid = e->row_valid;
+    gemm(e, &e->tm_zp, &e->tm_conv1_w, e->zp_alloc, e->mel_ld, e->conv1_w, 3L * e->mel_ld, p.total_prows, d,
+         3 * e->mel_ld, e->mel_ld, kEpiConv1, ep, s);
+  }
+  {
+    Prof pr(e, 2, s);
+    EpiParams ep{};
+    ep.bias = e->conv2_b; ep.resid = e->x; ep.ldc = d; ep.row_dst = e->row_dst; ep.pe = e->pe;
+    gemm(e, &e->tm_c1p, &e->tm_conv2_w, e->c1p, 2L * d, e->conv2_w, 3L * d, p.total_prows / 2, d, 3 * d, 2 * d,
+         kEpiConv2, ep, s);
+  }
+  for (int l = 0; l < c.n_layer; ++l) {
+    LayerW& w = e->layers[l];
+    {
+      Prof pr(e, 3, s);
+      launch_layernorm(e->x, w.ln1_g, w.ln1_b, e->h, bf, M, d, s);
+    }
+    {
+      Prof pr(e, 4, s);
+      EpiParams ep{};
+      ep.bias = w.bqkv; ep.out = e->qkv; ep.ldc = 3L * d;
+      gemm(e, &e->tm_h, &w.tm_wqkv, e->h, d, w.wqkv, d, M, 3 * d, d, d, kEpiBias, ep, s);
+    }
+    {
+      Prof pr(e, 5, s);
+      if (e->bf16) launch_attention_bf16((const __nv_bfloat16*)e->qkv, (__nv_bfloat16*)e->attn, meta, p.ml, p.n_work, d, s);
+      else launch_attention_f32((const float*)e->qkv, (float*)e->attn, meta, p.ml, p.n_work, d, s);
+    }
+    {
+      Prof pr(e, 4, s);
+      EpiParams ep{};
+      ep.bias = w.bo; ep.resid = e->x; ep.ldc = d;
+      gemm(e, &e->tm_attn, &w.tm_wo, e->attn, d, w.wo, d, M, d, d, d, kEpiBiasResid, ep, s);
+    }
+    {
+      Prof pr(e, 3, s);
+      launch_layernorm(e->x, w.ln2_g, w.ln2_b, e->h, bf, M, d, s);
+    }
+    {
+      Prof pr(e, 4, s);
+      EpiParams ep{};
+      ep.bias = w.b1; ep.out = e->fc1; ep.ldc = F;
+      gemm(e, &e->tm_h, &w.tm_w1, e->h, d, w.w1, d, M, F, d, d, kEpiBiasGelu, ep, s);
+    }
+    {
+      Prof pr(e, 4, s);
+      EpiParams ep{};
+      ep.bias = w.b2; ep.resid = e->x; ep.ldc = d;
+      gemm(e, &e->tm_fc1, &w.tm_w2, e->fc1, F, w.w2, F, M, d, F, F, kEpiBiasResid, ep, s);
+    }
+  }
+  {
+    Prof pr(e, 3, s);
+    launch_layernorm(e->x, e->lnp_g, e->lnp_b, hidden_out, bf, M, d, s);
+  }
+  WF_CUDA(e, cudaGetLastError());
+  return WF_OK;
+}
+
+wf_status encode_impl(wf_encoder* e, const float* audio, const float* mel, const long* len, int B,
+                      const float* hush, void* hidden_out, int* cu_out, cudaStream_t s) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  const wf_config& c = e->cfg;
+  if (c.hush_frames > 0 && !hush) return fail(e, WF_ERR_INVALID_ARG, "hush_mel is NULL but hush_frames > 0");
+  if (B > 0 && (!hidden_out || (!audio && !mel))) return fail(e, WF_ERR_INVALID_ARG, "NULL input or output");
+  if (B > c.max_batch) return fail(e, WF_ERR_CAPACITY, "batch %d exceeds max_batch %d", B, c.max_batch);
+  if (B < 0) return fail(e, WF_ERR_INVALID_ARG, "negative batch");
+  int slot;
+  wf_status st = ring_acquire(e, &slot);
+  if (st != WF_OK) return st;
+  Plan p;
+  st = make_plan(e, len, mel != nullptr, B, &p, e->meta_host[slot]);
+  if (st != WF_OK) return st;
+  if (cu_out)
+    for (int i = 0; i <= B; ++i) cu_out[i] = e->meta_host[slot][p.ml.tok_off + i];
+  if (B == 0) return WF_OK;
+  st = ring_upload(e, slot, p, s);
+  if (st != WF_OK) return st;
+  const int* meta = e->meta_dev[slot];
+  void* zp = (uint8_t*)e->zp_alloc + (size_t)e->mel_ld * e->esz;  // row 0 sits behind one guard row
+  if (audio) {
+    {
+      Prof pr(e, 0, s);
+      launch_fill_seq_max(e->seq_max, B, s);
+      launch_frontend(audio, meta, p.ml, B, p.n_fe_tiles, e->dft_basis, e->mel_fb_t, c.n_mel, e->logmel,
+                      e->seq_max, s);
+    }
+    {
+      Prof pr(e, 1, s);
+      launch_normalise(e->logmel, e->seq_max, nullptr, meta, p.ml, B, p.max_prows_seq, c.n_mel, e->mel_ld,
+                       c.hush_frames, hush, zp, e->bf16 ? 1 : 0, 1, s);
+    }
+  } else {
+    Prof pr(e, 1, s);
+    launch_normalise(nullptr, nullptr, mel, meta, p.ml, B, p.max_prows_seq, c.n_mel, e->mel_ld, c.hush_frames,
+                     hush, zp, e->bf16 ? 1 : 0, 1, s);
+  }
+  st = run_encoder(e, p, meta, hidden_out, s);
+  if (st != WF_OK) return st;
+  return ring_release(e, slot, s);
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+extern "C" {
+
+wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* stream, wf_encoder** out) {
+  if (!cfg || !w || !out) return WF_ERR_INVALID_ARG;
+  *out = nullptr;
+  cudaStream_t s = (cudaStream_t)stream;
+  wf_encoder* e = new (std::nothrow) wf_encoder();
+  if (!e) return WF_ERR_INVALID_ARG;
+  e->cfg = *cfg;
+  e->err[0] = 0;
+  e->profile = false;
+  e->prof_used = 0;
+  e->ring_pos = 0;
+  for (int i = 0; i < kRing; ++i) { e->meta_used[i] = false; e->meta_dev[i] = nullptr; e->meta_host[i] = nullptr; e->meta_ev[i] = nullptr; }
+  *out = e;  // returned even on failure so that the caller can read the message, then destroy
+  const wf_config& c = e->cfg;
+  if (c.n_mel <= 0 || c.n_mel % 8 || c.n_mel > 128 || c.d_model <= 0 || c.d_model % 128 || c.d_model > 1280 ||
+      c.n_head * kHeadDim != c.d_model || c.d_mlp <= 0 || c.d_mlp % 128 || c.n_layer < 0 || c.n_ctx < 1 ||
+      c.hush_frames < 0 || c.max_batch < 1 || c.max_tokens < 1 || c.max_samples < 0 ||
+      c.max_samples >= (1L << 31) - 1 || c.max_tokens > (1L << 28) || (c.dtype != WF_F32 && c.dtype != WF_BF16))
+    return fail(e, WF_ERR_INVALID_ARG, "unsupported configuration (see wf_config in wf_encoder.h)");
+  int dev = 0;
+  WF_CUDA(e, cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  WF_CUDA(e, cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return fail(e, WF_ERR_UNSUPPORTED_ARCH, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor);
+  e->num_sms = prop.multiProcessorCount;
+  e->bf16 = c.dtype == WF_BF16;
+  e->esz = e->bf16 ? 2 : 4;
+  e->mel_ld = e->bf16 ? (c.n_mel + 63) / 64 * 64 : c.n_mel;
+  e->cap_prows = 2 * (c.max_tokens + c.max_batch);
+  const int d = c.d_model, F = c.d_mlp;
+  wf_status st;
+#define WF_TRY(x) do { st = (x); if (st != WF_OK) return st; } while (0)
+
+  if (e->bf16) {
+    if (!tma_api_init(&e->tma)) return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    WF_CUDA(e, gemm_bf16_configure());
+    WF_CUDA(e, attention_bf16_configure());
+  }
+  // tables
+  WF_TRY(dev_alloc<float>(e, &e->dft_basis, 2L * kFold * kBasisCols));
+  WF_TRY(dev_alloc<float>(e, &e->pe, (size_t)c.n_ctx * d));
+  launch_build_tables(e->dft_basis, e->pe, c.n_ctx, d, s);
+  if (!w->mel_fb) return fail(e, WF_ERR_INVALID_ARG, "mel_fb is NULL");
+  WF_TRY(dev_alloc<float>(e, &e->mel_fb_t, (size_t)kBins * c.n_mel));
+  launch_transpose_f32(w->mel_fb, e->mel_fb_t, c.n_mel, kBins, s);
+  // conv stem
+  WF_TRY(dev_alloc_bytes(e, &e->conv1_w, (size_t)d * 3 * e->mel_ld * e->esz, true));
+  WF_TRY(dev_alloc_bytes(e, &e->conv2_w, (size_t)d * 3 * d * e->esz, true));
+  if (!w->conv1_w || !w->conv2_w) return fail(e, WF_ERR_INVALID_ARG, "conv weights are NULL");
+  launch_conv_weight(w->conv1_w, e->conv1_w, d, c.n_mel, e->mel_ld, e->bf16, s);
+  launch_conv_weight(w->conv2_w, e->conv2_w, d, d, d, e->bf16, s);
+  WF_TRY(own_f32(e, &e->conv1_b, w->conv1_b, d, s));
+  WF_TRY(own_f32(e, &e->conv2_b, w->conv2_b, d, s));
+  WF_TRY(own_f32(e, &e->lnp_g, w->lnp_g, d, s));
+  WF_TRY(own_f32(e, &e->lnp_b, w->lnp_b, d, s));
+  // blocks
+  e->layers.resize(c.n_layer);
+  if (c.n_layer > 0 && (!w->ln1_g || !w->ln1_b || !w->wq || !w->bq || !w->wk || !w->wv || !w->bv || !w->wo ||
+                        !w->bo || !w->ln2_g || !w->ln2_b || !w->w1 || !w->b1 || !w->w2 || !w->b2))
+    return fail(e, WF_ERR_INVALID_ARG, "a per-layer weight array is NULL");
+  for (int l = 0; l < c.n_layer; ++l) {
+    LayerW& L = e->layers[l];
+    WF_TRY(own_f32(e, &L.ln1_g, w->ln1_g[l], d, s));
+    WF_TRY(own_f32(e, &L.ln1_b, w->ln1_b[l], d, s));
+    WF_TRY(own_f32(e, &L.ln2_g, w->ln2_g[l], d, s));
+    WF_TRY(own_f32(e, &L.ln2_b, w->ln2_b[l], d, s));
+    WF_TRY(dev_alloc_bytes(e, &L.wqkv, (size_t)3 * d * d * e->esz));
+    WF_TRY(own_mat(e, L.wqkv, 0, w->wq[l], (size_t)d * d, s));
+    WF_TRY(own_mat(e, L.wqkv, (size_t)d * d, w->wk[l], (size_t)d * d, s));
+    WF_TRY(own_mat(e, L.wqkv, (size_t)2 * d * d, w->wv[l], (size_t)d * d, s));
+    WF_TRY(dev_alloc<float>(e, &L.bqkv, 3 * d, true));  // the key part stays zero
+    if (!w->bq[l] || !w->bv[l]) return fail(e, WF_ERR_INVALID_ARG, "a bias pointer is NULL");
+    WF_CUDA(e, cudaMemcpyAsync(L.bqkv, w->bq[l], d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    WF_CUDA(e, cudaMemcpyAsync(L.bqkv + 2 * d, w->bv[l], d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    WF_TRY(dev_alloc_bytes(e, &L.wo, (size_t)d * d * e->esz));
+    WF_TRY(own_mat(e, L.wo, 0, w->wo[l], (size_t)d * d, s));
+    WF_TRY(own_f32(e, &L.bo, w->bo[l], d, s));
+    WF_TRY(dev_alloc_bytes(e, &L.w1, (size_t)F * d * e->esz));
+    WF_TRY(own_mat(e, L.w1, 0, w->w1[l], (size_t)F * d, s));
+    WF_TRY(own_f32(e, &L.b1, w->b1[l], F, s));
+    WF_TRY(dev_alloc_bytes(e, &L.w2, (size_t)d * F * e->esz));
+    WF_TRY(own_mat(e, L.w2, 0, w->w2[l], (size_t)d * F, s));
+    WF_TRY(own_f32(e, &L.b2, w->b2[l], d, s));
+  }
+  // workspace
+  const size_t mt = (size_t)c.max_tokens;
+  WF_TRY(dev_alloc<float>(e, &e->logmel, (size_t)(c.max_samples / kHop + 1) * c.n_mel));
+  WF_TRY(dev_alloc<int>(e, &e->seq_max, c.max_batch));
+  WF_TRY(dev_alloc_bytes(e, &e->zp_alloc, (size_t)(e->cap_prows + 4) * e->mel_ld * e->esz, true));
+  WF_TRY(dev_alloc_bytes(e, &e->c1p, (size_t)(e->cap_prows + 4) * d * e->esz, true));
+  WF_TRY(dev_alloc<int>(e, &e->row_valid, (size_t)e->cap_prows + 4, true));
+  WF_TRY(dev_alloc<int2>(e, &e->row_dst, (size_t)e->cap_prows / 2 + 4, true));
+  WF_TRY(dev_alloc<float>(e, &e->x, mt * d));
+  WF_TRY(dev_alloc_bytes(e, &e->h, mt * d * e->esz, true));
+  WF_TRY(dev_alloc_bytes(e, &e->qkv, mt * 3 * d * e->esz, true));
+  WF_TRY(dev_alloc_bytes(e, &e->attn, mt * d * e->esz, true));
+  WF_TRY(dev_alloc_bytes(e, &e->fc1, mt * F * e->esz, true));
+  WF_TRY(dev_alloc<float>(e, &e->audio_stage, (size_t)c.max_samples));
+  WF_TRY(dev_alloc_bytes(e, &e->out_stage, mt * d * e->esz));
+  WF_TRY(dev_alloc<int>(e, &e->err_flag, 1, true));
+  e->meta_cap = 6 * (c.max_batch + 1) + 2 * (int)(c.max_tokens / 16 + c.max_batch) + 16;
+  for (int i = 0; i < kRing; ++i) {
+    WF_TRY(dev_alloc<int>(e, &e->meta_dev[i], e->meta_cap));
+    void* hp = nullptr;
+    WF_CUDA(e, cudaMallocHost(&hp, (size_t)e->meta_cap * sizeof(int)));
+    e->pinned.push_back(hp);
+    e->meta_host[i] = (int*)hp;
+    WF_CUDA(e, cudaEventCreateWithFlags(&e->meta_ev[i], cudaEventDisableTiming));
+  }
+  if (e->bf16) {
+    bool ok = true;
+    ok &= make_tmap_bf16(e->tma, &e->tm_zp, e->zp_alloc, e->mel_ld, e->cap_prows + 4, e->mel_ld, 128);
+    ok &= make_tmap_bf16(e->tma, &e->tm_c1p, e->c1p, 2 * d, (e->cap_prows + 4) / 2, 2 * d, 128);
+    ok &= make_tmap_bf16(e->tma, &e->tm_h, e->h, d, mt, d, 128);
+    ok &= make_tmap_bf16(e->tma, &e->tm_attn, e->attn, d, mt, d, 128);
+    ok &= make_tmap_bf16(e->tma, &e->tm_fc1, e->fc1, F, mt, F, 128);
+    ok &= make_tmap_bf16(e->tma, &e->tm_conv1_w, e->conv1_w, 3 * e->mel_ld, d, 3 * e->mel_ld, 256);
+    ok &= make_tmap_bf16(e->tma, &e->tm_conv2_w, e->conv2_w, 3 * d, d, 3 * d, 256);
+    for (int l = 0; l < c.n_layer; ++l) {
+      LayerW& L = e->layers[l];
+      ok &= make_tmap_bf16(e->tma, &L.tm_wqkv, L.wqkv, d, 3 * d, d, 256);
+      ok &= make_tmap_bf16(e->tma, &L.tm_wo, L.wo, d, d, d, 256);
+      ok &= make_tmap_bf16(e->tma, &L.tm_w1, L.w1, d, F, d, 256);
+      ok &= make_tmap_bf16(e->tma, &L.tm_w2, L.w2, F, d, F, 256);
+    }
+    if (!ok) return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
+  }
+  WF_CUDA(e, cudaGetLastError());
+  WF_CUDA(e, cudaStreamSynchronize(s));
+#undef WF_TRY
+  return WF_OK;
+}
+
+wf_status wf_encoder_destroy(wf_encoder* e) {
+  if (!e) return WF_OK;
+  cudaDeviceSynchronize();
+  for (void* p : e->allocs) cudaFree(p);
+  for (void* p : e->pinned) cudaFreeHost(p);
+  for (int i = 0; i < kRing; ++i)
+    if (e->meta_ev[i]) cudaEventDestroy(e->meta_ev[i]);
+  for (auto& pe : e->prof) { cudaEventDestroy(pe.a); cudaEventDestroy(pe.b); }
+  delete e;
+  return WF_OK;
+}
+
+const char* wf_last_error(const wf_encoder* e) { return e ? e->err : "null encoder"; }
+
+wf_status wf_logmel(wf_encoder* e, const float* audio, const long* lengths, int B, float* mel_out,
+                    long* frames_out, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (B > 0 && (!audio || !mel_out)) return fail(e, WF_ERR_INVALID_ARG, "NULL audio or output");
+  if (B > e->cfg.max_batch) return fail(e, WF_ERR_CAPACITY, "batch %d exceeds max_batch %d", B, e->cfg.max_batch);
+  if (B < 0) return fail(e, WF_ERR_INVALID_ARG, "negative batch");
+  int slot;
+  wf_status st = ring_acquire(e, &slot);
+  if (st != WF_OK) return st;
+  Plan p;
+  // frame counts do not depend on the hush length; token limits do not apply to the front end
+  wf_config saved = e->cfg;
+  e->cfg.hush_frames = 0;
+  e->cfg.n_ctx = 1 << 28;
+  e->cfg.max_tokens = 1L << 40;
+  st = make_plan(e, lengths, false, B, &p, e->meta_host[slot], false);
+  e->cfg = saved;
+  if (st != WF_OK) return st;
+  if (frames_out)
+    for (int i = 0; i < B; ++i) frames_out[i] = e->meta_host[slot][p.ml.frames + i];
+  if (B == 0) return WF_OK;
+  p.ml.total = p.ml.attn_work;  // no attention work list needed
+  st = ring_upload(e, slot, p, s);
+  if (st != WF_OK) return st;
+  const int* meta = e->meta_dev[slot];
+  int max_T = 0;
+  for (int i = 0; i < B; ++i) max_T = std::max(max_T, e->meta_host[slot][p.ml.frames + i]);
+  {
+    Prof pr(e, 0, s);
+    launch_fill_seq_max(e->seq_max, B, s);
+    launch_frontend(audio, meta, p.ml, B, p.n_fe_tiles, e->dft_basis, e->mel_fb_t, e->cfg.n_mel, e->logmel,
+                    e->seq_max, s);
+  }
+  {
+    Prof pr(e, 1, s);
+    launch_normalise(e->logmel, e->seq_max, nullptr, meta, p.ml, B, max_T, e->cfg.n_mel, e->cfg.n_mel, 0, nullptr,
+                     mel_out, 0, 0, s);
+  }
+  WF_CUDA(e, cudaGetLastError());
+  return ring_release(e, slot, s);
+}
+
+wf_status wf_encode(wf_encoder* e, const float* audio, const long* lengths, int B, const float* hush_mel,
+                    void* hidden_out, int* cu_seqlens_out, void* stream) {
+  return encode_impl(e, audio, nullptr, lengths, B, hush_mel, hidden_out, cu_seqlens_out, (cudaStream_t)stream);
+}
+
+wf_status wf_encode_mel(wf_encoder* e, const float* mel, const long* frames, int B, const float* hush_mel,
+                        void* hidden_out, int* cu_seqlens_out, void* stream) {
+  return encode_impl(e, nullptr, mel, frames, B, hush_mel, hidden_out, cu_seqlens_out, (cudaStream_t)stream);
+}
+
+wf_status wf_encode_host(wf_encoder* e, const float* audio_host, const long* lengths, int B,
+                         const float* hush_mel, void* hidden_out_host, int* cu_seqlens_out, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (B < 0 || (B > 0 && (!audio_host || !lengths || !hidden_out_host)))
+    return fail(e, WF_ERR_INVALID_ARG, "NULL input or output");
+  long total = 0;
+  for (int i = 0; i < B; ++i) {
+    if (lengths[i] < 0) return fail(e, WF_ERR_INVALID_ARG, "negative length");
+    total += lengths[i];
+    if (total > e->cfg.max_samples) return fail(e, WF_ERR_CAPACITY, "more than max_samples=%ld samples", e->cfg.max_samples);
+  }
+  if (total > 0) WF_CUDA(e, cudaMemcpyAsync(e->audio_stage, audio_host, (size_t)total * sizeof(float), cudaMemcpyHostToDevice, s));
+  std::vector<int> cu(B + 1, 0);
+  wf_status st = encode_impl(e, e->audio_stage, nullptr, lengths, B, hush_mel, e->out_stage, cu.data(), s);
+  if (st != WF_OK) return st;
+  if (cu_seqlens_out) std::memcpy(cu_seqlens_out, cu.data(), (size_t)(B + 1) * sizeof(int));
+  size_t bytes = (size_t)cu[B] * e->cfg.d_model * e->esz;
+  if (bytes) WF_CUDA(e, cudaMemcpyAsync(hidden_out_host, e->out_stage, bytes, cudaMemcpyDeviceToHost, s));
+  WF_CUDA(e, cudaStreamSynchronize(s));
+  return WF_OK;
+}
+
+wf_status wf_check(wf_encoder* e, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  WF_CUDA(e, cudaStreamSynchronize(s));
+  int flag = 0;
+  WF_CUDA(e, cudaMemcpy(&flag, e->err_flag, sizeof(int), cudaMemcpyDeviceToHost));
+  if (flag != 0) {
+    cudaMemset(e->err_flag, 0, sizeof(int));
+    return fail(e, WF_ERR_DEVICE_TIMEOUT, "a bounded wait inside a GEMM kernel gave up (role %d)", flag);
+  }
+  return WF_OK;
+}
+
+wf_status wf_profile_enable(wf_encoder* e, int on) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  e->profile = on != 0;
+  return WF_OK;
+}
+
+wf_status wf_profile_read(wf_encoder* e, long* launches, double* millis) {
+  if (!e || !launches || !millis) return WF_ERR_INVALID_ARG;
+  WF_CUDA(e, cudaDeviceSynchronize());
+  for (int c = 0; c < WF_N_KERNEL_CLASSES; ++c) { launches[c] = 0; millis[c] = 0.0; }
+  for (size_t i = 0; i < e->prof_used; ++i) {
+    float ms = 0.f;
+    WF_CUDA(e, cudaEventElapsedTime(&ms, e->prof[i].a, e->prof[i].b));
+    launches[e->prof[i].cls] += 1;
+    millis[e->prof[i].cls] += ms;
+  }
+  e->prof_used = 0;
+  return WF_OK;
+}
+
+wf_status wf_gemm_bf16(wf_encoder* e, const void* A, const void* W, const float* bias, void* C, long M, int N,
+                       int K, int mode, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  if (!e->bf16) return fail(e, WF_ERR_INVALID_ARG, "wf_gemm_bf16 needs an encoder created with WF_BF16");
+  if (!A || !W || !bias || !C || M < 0 || N <= 0 || K <= 0 || N % 8 || K % 8 || mode < 0 || mode > 2 ||
+      ((uintptr_t)A & 15) || ((uintptr_t)W & 15) || ((uintptr_t)C & 15) || ((uintptr_t)bias & 15))
+    return fail(e, WF_ERR_INVALID_ARG, "wf_gemm_bf16: bad pointer, size or mode");
+  if (M == 0) return WF_OK;
+  CUtensorMap ta, tb;
+  if (!make_tmap_bf16(e->tma, &ta, A, K, M, K, 128) || !make_tmap_bf16(e->tma, &tb, W, K, N, K, 256))
+    return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
+  EpiParams ep{};
+  ep.bias = bias;
+  ep.ldc = N;
+  if (mode == 2) ep.resid = (float*)C; else ep.out = C;
+  launch_gemm_bf16(ta, tb, M, N, K, K, mode, ep, e->err_flag, e->num_sms, (cudaStream_t)stream);
+  WF_CUDA(e, cudaGetLastError());
+  return WF_OK;
+}
+
+wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, int B, void* out, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (B < 0 || (B > 0 && (!qkv || !cu_seqlens || !out))) return fail(e, WF_ERR_INVALID_ARG, "NULL argument");
+  if (B > e->cfg.max_batch) return fail(e, WF_ERR_CAPACITY, "batch %d exceeds max_batch %d", B, e->cfg.max_batch);
+  if (B == 0) return WF_OK;
+  if (cu_seqlens[0] != 0) return fail(e, WF_ERR_INVALID_ARG, "cu_seqlens[0] must be 0");
+  for (int i = 0; i < B; ++i)
+    if (cu_seqlens[i + 1] <= cu_seqlens[i]) return fail(e, WF_ERR_INVALID_ARG, "cu_seqlens must increase strictly");
+  if (cu_seqlens[B] > e->cfg.max_tokens) return fail(e, WF_ERR_CAPACITY, "more than max_tokens tokens");
+  int slot;
+  wf_status st = ring_acquire(e, &slot);
+  if (st != WF_OK) return st;
+  int* hm = e->meta_host[slot];
+  MetaLayout ml{};
+  ml.tok_off = 0;
+  ml.attn_work = B + 1;
+  for (int i = 0; i <= B; ++i) hm[i] = cu_seqlens[i];
+  const int qt = e->bf16 ? 64 : 16;
+  int nw = 0;
+  for (int i = 0; i < B; ++i)
+    for (int q0 = 0; q0 < cu_seqlens[i + 1] - cu_seqlens[i]; q0 += qt) {
+      hm[ml.attn_work + 2 * nw] = i;
+      hm[ml.attn_work + 2 * nw + 1] = q0;
+      ++nw;
+    }
+  ml.total = ml.attn_work + 2 * nw;
+  Plan p{};
+  p.ml = ml;
+  st = ring_upload(e, slot, p, s);
+  if (st != WF_OK) return st;
+  {
+    Prof pr(e, 5, s);
+    if (e->bf16) launch_attention_bf16((const __nv_bfloat16*)qkv, (__nv_bfloat16*)out, e->meta_dev[slot], ml, nw, e->cfg.d_model, s);
+    else launch_attention_f32((const float*)qkv, (float*)out, e->meta_dev[slot], ml, nw, e->cfg.d_model, s);
+  }
+  WF_CUDA(e, cudaGetLastError());
+  return ring_release(e, slot, s);
+}
+
+}  // extern "C"

@@ -142,7 +142,7 @@ void launch_layernorm(const float* x, const float* g, const float* b, void* out,
 }
 
 // ---------------------------------------------------------------------------------------------
-// float32 attention: one CTA = 32 queries of one (sequence, head); 8 warps x 4 queries.  Keys
+// float32 attention: one CTA = 16 queries of one (sequence, head); 8 warps x 2 queries.  Keys
 // and values are staged 64 at a time; scores are lane-per-key, outputs lane-per-channel.
 __global__ void __launch_bounds__(256) attention_f32_kernel(const float* __restrict__ qkv,
                                                             float* __restrict__ out,
@@ -150,8 +150,8 @@ __global__ void __launch_bounds__(256) attention_f32_kernel(const float* __restr
                                                             MetaLayout ml, int d_model) {
   __shared__ float Ks[64][65];
   __shared__ float Vs[64][64];
-  __shared__ float Qs[32][64];
-  __shared__ float Ps[8][4][64];
+  __shared__ float Qs[16][64];
+  __shared__ float Ps[8][2][64];
   const int seq = meta[ml.attn_work + 2 * blockIdx.x];
   const int q0 = meta[ml.attn_work + 2 * blockIdx.x + 1];
   const int head = blockIdx.y;
@@ -163,13 +163,13 @@ __global__ void __launch_bounds__(256) attention_f32_kernel(const float* __restr
   const float* kb = qb + d_model;
   const float* vb = qb + 2 * d_model;
 
-  for (int i = tid; i < 32 * 64; i += 256) {
+  for (int i = tid; i < 16 * 64; i += 256) {
     int r = i >> 6, c = i & 63;
     Qs[r][c] = (q0 + r < n) ? qb[(long)(q0 + r) * ld + c] * 0.125f : 0.f;
   }
-  float m_run[4], l_run[4], o0[4], o1[4];
+  float m_run[2], l_run[2], o0[2], o1[2];
 #pragma unroll
-  for (int qi = 0; qi < 4; ++qi) { m_run[qi] = -INFINITY; l_run[qi] = 0.f; o0[qi] = 0.f; o1[qi] = 0.f; }
+  for (int qi = 0; qi < 2; ++qi) { m_run[qi] = -INFINITY; l_run[qi] = 0.f; o0[qi] = 0.f; o1[qi] = 0.f; }
 
   for (int k0 = 0; k0 < n; k0 += 64) {
     __syncthreads();
@@ -180,20 +180,20 @@ __global__ void __launch_bounds__(256) attention_f32_kernel(const float* __restr
       Vs[r][c] = ok ? vb[(long)(k0 + r) * ld + c] : 0.f;
     }
     __syncthreads();
-    float sc[4][2];
+    float sc[2][2];
 #pragma unroll
-    for (int qi = 0; qi < 4; ++qi) { sc[qi][0] = 0.f; sc[qi][1] = 0.f; }
+    for (int qi = 0; qi < 2; ++qi) { sc[qi][0] = 0.f; sc[qi][1] = 0.f; }
     for (int c = 0; c < 64; ++c) {
       float ka = Ks[lane][c], kb2 = Ks[lane + 32][c];
 #pragma unroll
-      for (int qi = 0; qi < 4; ++qi) {
-        float qv = Qs[warp * 4 + qi][c];
+      for (int qi = 0; qi < 2; ++qi) {
+        float qv = Qs[warp * 2 + qi][c];
         sc[qi][0] = fmaf(qv, ka, sc[qi][0]);
         sc[qi][1] = fmaf(qv, kb2, sc[qi][1]);
       }
     }
 #pragma unroll
-    for (int qi = 0; qi < 4; ++qi) {
+    for (int qi = 0; qi < 2; ++qi) {
       if (k0 + lane >= n) sc[qi][0] = -INFINITY;
       if (k0 + lane + 32 >= n) sc[qi][1] = -INFINITY;
       float mx = fmaxf(sc[qi][0], sc[qi][1]);
@@ -215,7 +215,7 @@ __global__ void __launch_bounds__(256) attention_f32_kernel(const float* __restr
     for (int key = 0; key < 64; ++key) {
       float v0 = Vs[key][lane], v1 = Vs[key][lane + 32];
 #pragma unroll
-      for (int qi = 0; qi < 4; ++qi) {
+      for (int qi = 0; qi < 2; ++qi) {
         float p = Ps[warp][qi][key];
         o0[qi] = fmaf(p, v0, o0[qi]);
         o1[qi] = fmaf(p, v1, o1[qi]);
@@ -224,8 +224,8 @@ __global__ void __launch_bounds__(256) attention_f32_kernel(const float* __restr
     __syncwarp();
   }
 #pragma unroll
-  for (int qi = 0; qi < 4; ++qi) {
-    int q = q0 + warp * 4 + qi;
+  for (int qi = 0; qi < 2; ++qi) {
+    int q = q0 + warp * 2 + qi;
     if (q < n) {
       float inv = 1.0f / l_run[qi];
       float* orow = out + (long)(tok0 + q) * d_model + head * kHeadDim;

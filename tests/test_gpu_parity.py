@@ -1,0 +1,274 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 oracle on the same
+seeded inputs.  Tolerances: float32 path max-abs <= 1e-3 on final hidden states; bf16 path
+max|err| / max|ref| <= 3e-2 per sequence and per-token cosine >= 0.999."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import wf_oracle as O
+from paper_2412_11272_b200 import inputs as I
+from tests._util import make_encoder, min_token_cosine, oracle_hidden, peak_rel_err, to_np
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+F32_TOL = 1e-3
+BF16_REL, BF16_COS = 3e-2, 0.999
+MEL_TOL = 2e-4   # normalised log-mel units; float32 DFT of 400 terms under a log10
+
+
+def _dev(a, dtype=torch.float32):
+    return torch.as_tensor(np.ascontiguousarray(a)).to("cuda:0", dtype)
+
+
+def _small(dtype, **kw):
+    base = dict(name="s", n_mel=80, d_model=128, n_layer=2, n_head=2, d_mlp=256, dtype=dtype, n_ctx=1536)
+    base.update(kw)
+    return I.EncoderShape(**base)
+
+
+# ------------------------------------------------------------------------------ front end
+
+def test_logmel_matches_oracle_ragged():
+    shape = _small("f32", n_layer=0)
+    W = I.encoder_weights(0, shape)
+    lengths = [32000, 401, 160 * 64, 160 * 65 + 37, 160 * 129 + 159, 5000]
+    batch = I.batch_from_lengths(11, lengths)
+    enc = make_encoder(shape, W, 8, 4096, int(sum(lengths)))
+    mel, frames = enc.wf_logmel(_dev(batch.audio), batch.lengths)
+    torch.cuda.synchronize()
+    assert list(frames) == [n // 160 for n in lengths]
+    got = to_np(mel)
+    F = I.mel_filterbank(80)
+    off = 0
+    for s in batch.sequences():
+        ref = O.log_mel(s, F)
+        g = got[off:off + ref.shape[0]]
+        off += ref.shape[0]
+        assert np.max(np.abs(g - ref)) < MEL_TOL
+    assert off == got.shape[0]
+    enc.close()
+
+
+def test_logmel_pure_sine_and_silence():
+    shape = _small("f32", n_layer=0)
+    enc = make_encoder(shape, I.encoder_weights(0, shape), 2, 1024, 40000)
+    t = np.arange(16000)
+    sine = (0.5 * np.sin(2 * math.pi * 1000.0 * t / 16000)).astype(np.float32)
+    silence = np.zeros(8000, np.float32)
+    mel, _ = enc.wf_logmel(_dev(np.concatenate([sine, silence])), [16000, 8000])
+    got = to_np(mel)
+    F = I.mel_filterbank(80)
+    centre = np.argmax(F, axis=1) * 40.0
+    assert np.argmax(got[50]) == np.argmin(np.abs(centre - 1000.0))
+    assert np.allclose(got[100:], -1.5, atol=1e-6)          # (log10(1e-10) + 4) / 4
+    enc.close()
+
+
+# ------------------------------------------------------------------------------ float32 path
+
+def test_f32_tiny_config_matches_oracle():
+    """The smallest configuration: tiny-shaped float32 encoder, one 2.0 s buffer + 50 hush frames."""
+    shape = I.SHAPES["tiny"]
+    W = I.encoder_weights(0, shape)
+    batch = I.config_batch("tiny")
+    hush = I.hush_mel(0, shape.n_mel)
+    enc = make_encoder(shape, W, 1, 125, 32000)
+    out, cu = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush))
+    enc.wf_check()
+    assert list(cu) == [0, 125] and out.shape == (125, 384) and out.dtype == torch.float32
+    ref = oracle_hidden(batch, shape, W, hush)[0]
+    assert np.max(np.abs(to_np(out) - ref)) <= F32_TOL
+    enc.close()
+
+
+def test_f32_ragged_batch_odd_even_and_invariance():
+    shape = _small("f32")
+    W = I.encoder_weights(3, shape, logit_gain=12.0)
+    lengths = [160 * 7, 160 * 10, 401, 160 * 131, 160 * 64 + 5]      # T' odd and even, tiny, multi-tile
+    batch = I.batch_from_lengths(5, lengths)
+    hush = I.hush_mel(5, shape.n_mel, 3)
+    enc = make_encoder(shape, W, 8, 512, int(sum(lengths)), hush_frames=3)
+    out, cu = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush))
+    enc.wf_check()
+    got = to_np(out)
+    F = I.mel_filterbank(shape.n_mel)
+    refs = [O.encode_sequence(s, F, hush, W, shape.n_layer, shape.n_head) for s in batch.sequences()]
+    assert list(cu) == list(np.concatenate([[0], np.cumsum([r.shape[0] for r in refs])]))
+    for i, r in enumerate(refs):
+        assert np.max(np.abs(got[cu[i]:cu[i + 1]] - r)) <= F32_TOL, i
+    # batch invariance: a sequence alone, or in another order, gives the same rows
+    order = [3, 0, 4]
+    b2 = I.Batch(np.concatenate([batch.sequences()[i] for i in order]), batch.lengths[order])
+    out2, cu2 = enc.wf_encode(_dev(b2.audio), b2.lengths, _dev(hush))
+    g2 = to_np(out2)
+    for j, i in enumerate(order):
+        assert np.max(np.abs(g2[cu2[j]:cu2[j + 1]] - got[cu[i]:cu[i + 1]])) <= 1e-5
+    enc.close()
+
+
+def test_encode_mel_entry_and_raw_audio_level_hush():
+    """The paper attaches the hush word at raw-audio level: the caller concatenates samples and
+    runs with hush_frames = 0; wf_encode_mel consumes rows made by wf_logmel."""
+    shape = _small("f32")
+    W = I.encoder_weights(4, shape)
+    x = I.synth_audio(6, 0, 160 * 40)
+    h = I.hush_audio(6)
+    xa = np.concatenate([x, h]).astype(np.float32)
+    enc = make_encoder(shape, W, 2, 256, len(xa), hush_frames=0)
+    out, cu = enc.wf_encode(_dev(xa), [len(xa)], None)
+    ref = O.encode_sequence(x, I.mel_filterbank(80), h, W, shape.n_layer, shape.n_head, hush_level="audio")
+    assert list(cu) == [0, 45] and np.max(np.abs(to_np(out) - ref)) <= F32_TOL
+    mel, frames = enc.wf_logmel(_dev(xa), [len(xa)])
+    out2, _ = enc.wf_encode_mel(mel, frames, None)
+    assert np.max(np.abs(to_np(out2) - to_np(out))) <= 1e-6
+    enc.close()
+
+
+# ------------------------------------------------------------------------------ bf16 components
+
+@pytest.mark.parametrize("M,N,K", [(300, 384, 240), (1000, 1536, 512), (129, 256, 64), (4097, 1280, 1280),
+                                   (77, 8, 8)])
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_tcgen05_gemm_matches_fp64(M, N, K, mode):
+    shape = _small("bf16", n_layer=0)
+    enc = make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000)
+    rng = np.random.default_rng(M + N + K + mode)
+    A = I.round_to_bf16(rng.normal(size=(M, K)).astype(np.float32))
+    Wm = I.round_to_bf16((rng.normal(size=(N, K)) / math.sqrt(K)).astype(np.float32))
+    bias = rng.normal(size=N).astype(np.float32)
+    ref = A.astype(np.float64) @ Wm.astype(np.float64).T + bias
+    dA, dW, db = _dev(A, torch.bfloat16), _dev(Wm, torch.bfloat16), _dev(bias)
+    if mode == 2:
+        resid = rng.normal(size=(M, N)).astype(np.float32)
+        C = _dev(resid)
+        enc.wf_gemm_bf16(dA, dW, db, 2, C)
+        enc.wf_check()
+        assert np.max(np.abs(to_np(C) - (ref + resid))) < 2e-5 * math.sqrt(K) + 1e-5
+    else:
+        if mode == 1:
+            ref = O.gelu(ref)
+        C = enc.wf_gemm_bf16(dA, dW, db, mode)
+        enc.wf_check()
+        got = to_np(C)
+        assert np.max(np.abs(got - ref) / (np.abs(ref) + 1.0)) < 2.0 ** -8     # bf16 output rounding
+    enc.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_varlen_attention_matches_oracle(dtype):
+    shape = _small(dtype, n_layer=0, d_model=256, n_head=4, d_mlp=256)
+    enc = make_encoder(shape, I.encoder_weights(0, shape), 8, 4096, 1000)
+    lens = [1, 63, 64, 65, 200, 1525, 17]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    rng = np.random.default_rng(9)
+    qkv = rng.normal(size=(cu[-1], 3 * 256)).astype(np.float32)
+    qkv[:, :256] *= 3.0                                     # logits with std ~ 3: softmax far from uniform
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    if dtype == "bf16":
+        qkv = I.round_to_bf16(qkv)
+    out = to_np(enc.wf_attention(_dev(qkv, tdt), cu))
+    enc.wf_check()
+    q64 = qkv.astype(np.float64)
+    tol = 2e-2 if dtype == "bf16" else 1e-5
+    for i in range(len(lens)):
+        s = slice(cu[i], cu[i + 1])
+        ref = O.attention(q64[s, :256], q64[s, 256:512], q64[s, 512:], 4)
+        assert np.max(np.abs(out[s] - ref)) < tol, (i, lens[i])
+    # identical keys -> mean of values
+    q2 = qkv.copy()
+    q2[:, 256:512] = q2[0, 256:512]
+    out2 = to_np(enc.wf_attention(_dev(q2, tdt), cu))
+    s = slice(cu[4], cu[5])
+    assert np.max(np.abs(out2[s] - q2[s, 512:].astype(np.float64).mean(axis=0))) < tol
+    enc.close()
+
+
+# ------------------------------------------------------------------------------ bf16 path
+
+def _check_bf16(got, ref):
+    assert peak_rel_err(got, ref) <= BF16_REL
+    assert min_token_cosine(got, ref) >= BF16_COS
+
+
+def test_bf16_small_ragged_matches_oracle():
+    shape = _small("bf16", d_model=256, n_head=4, d_mlp=1024, n_layer=3)
+    W = I.encoder_weights(7, shape)
+    lengths = [160 * 7, 160 * 300, 401, 160 * 131, 160 * 64 + 5, 160 * 10]
+    batch = I.batch_from_lengths(8, lengths)
+    hush = I.round_to_bf16(I.hush_mel(8, shape.n_mel))
+    enc = make_encoder(shape, W, 8, 2048, int(sum(lengths)))
+    out, cu = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush))
+    enc.wf_check()
+    assert out.dtype == torch.bfloat16
+    got = to_np(out)
+    refs = oracle_hidden(batch, shape, W, hush)
+    for i, r in refs.items():
+        _check_bf16(got[cu[i]:cu[i + 1]], r)
+    enc.close()
+
+
+def test_bf16_attention_stress_weights():
+    """Query/key weights scaled so that logits have a standard deviation of a few units."""
+    shape = _small("bf16", d_model=256, n_head=4, d_mlp=512, n_layer=2)
+    W = I.encoder_weights(9, shape, logit_gain=6.0)
+    batch = I.batch_from_lengths(10, [160 * 250, 160 * 33])
+    hush = I.round_to_bf16(I.hush_mel(10, shape.n_mel))
+    enc = make_encoder(shape, W, 2, 1024, int(batch.lengths.sum()))
+    out, cu = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush))
+    enc.wf_check()
+    got = to_np(out)
+    for i, r in oracle_hidden(batch, shape, W, hush).items():
+        _check_bf16(got[cu[i]:cu[i + 1]], r)
+    enc.close()
+
+
+def test_bf16_base_config_matches_oracle():
+    """Base-shaped encoder, 16 buffers of 1-10 s + hush, ragged (the second configuration)."""
+    shape = I.SHAPES["base"]
+    W = I.encoder_weights(1, shape)
+    batch = I.config_batch("base")
+    hush = I.round_to_bf16(I.hush_mel(1, shape.n_mel))
+    M = int(I.tokens_of(batch.lengths).sum())
+    enc = make_encoder(shape, W, 16, M, int(batch.lengths.sum()))
+    out, cu = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush))
+    enc.wf_check()
+    got = to_np(out)
+    assert cu[-1] == M
+    for i, r in oracle_hidden(batch, shape, W, hush).items():
+        _check_bf16(got[cu[i]:cu[i + 1]], r)
+    # host-buffer entry point gives the same result
+    a_host = torch.as_tensor(batch.audio).pin_memory()
+    o_host = torch.empty((M, shape.d_model), dtype=torch.bfloat16).pin_memory()
+    enc.wf_encode_host(a_host, batch.lengths, _dev(hush), o_host)
+    assert torch.equal(o_host, out.cpu())
+    enc.close()
+
+
+# ------------------------------------------------------------------------------ errors and edges
+
+def test_errors_and_edge_cases():
+    from paper_2412_11272_b200.binding import WfError
+    shape = _small("f32", n_layer=1, n_ctx=40)
+    W = I.encoder_weights(2, shape)
+    enc = make_encoder(shape, W, 2, 64, 20000, hush_frames=3)
+    hush = _dev(I.hush_mel(2, 80, 3))
+    audio = _dev(I.synth_audio(2, 0, 20000))
+    out, cu = enc.wf_encode(audio, [], hush)                          # empty batch
+    assert list(cu) == [0] and out.shape[0] == 0
+    for lengths, status in (([400], "WF_ERR_TOO_SHORT"), ([160 * 80], "WF_ERR_TOO_LONG"),
+                            ([1000, 1000, 1000], "WF_ERR_CAPACITY"), ([10000, 10001], "WF_ERR_CAPACITY")):
+        with pytest.raises(WfError) as ei:
+            enc.wf_encode(audio, lengths, hush)
+        assert ei.value.status == status, lengths
+    with pytest.raises(WfError) as ei:
+        enc.wf_encode(audio, [1600], None)                            # hush required
+    assert ei.value.status == "WF_ERR_INVALID_ARG"
+    out, cu = enc.wf_encode(audio, [160 * 77], hush)                  # exactly n_ctx tokens is fine
+    assert cu[-1] == 40
+    enc.wf_check()
+    enc.close()
+    bad = I.EncoderShape("bad", 80, 96, 1, 2, 256, "f32")
+    with pytest.raises(WfError):
+        make_encoder(bad, I.encoder_weights(0, bad), 1, 8, 1000)
