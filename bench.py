@@ -1,0 +1,321 @@
+#!/usr/bin/env python
+"""Benchmark of the hush-terminated ragged encoder on the large-v3-shaped workload.
+
+One step = the sliding-window workload of 64 concurrent streams: 15 calls of ``wf_encode``,
+call k encoding all 64 streams' first k seconds (k = 1..15) plus the 50-frame hush segment as
+one ragged batch.  Audio-seconds count real audio only; tokens include the hush tokens.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Under torchrun every rank runs the same workload on its own streams (weak scaling, no
+data-path collective).  ``--impl reference`` times the fp64 CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2412_11272_b200 import inputs as I  # noqa: E402
+
+METRIC = "encoded_audio_seconds_per_sec"
+UNIT = "audio-s/s"
+WORKLOAD = "large-v3-shaped bf16 encoder, 64 streams x windows of 1..15 s + 50 hush frames (15 ragged calls per step)"
+N_STREAMS = 64
+ROUNDS = list(range(1, 16))
+SAMPLE_SECONDS = 15         # the CPU oracle is timed on stream 0's full 15 s window (775 tokens)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"],
+                "bf16_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake"}
+
+    def __init__(self, device_index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            import torch
+            uuid = getattr(torch.cuda.get_device_properties(device_index), "uuid", None)
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                try:
+                    mask = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop_evt.wait(0.1)
+
+    def finish(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_sample(weights, mel_fb, hush, seed, stream=0):
+    """The bounded CPU sample: stream `stream`'s first SAMPLE_SECONDS seconds through the oracle."""
+    from oracle import wf_oracle as O
+    shape = I.SHAPES["large"]
+    x = I.large_stream(seed, stream)[: SAMPLE_SECONDS * I.SAMPLE_RATE]
+    t0 = time.perf_counter()
+    ref = O.encode_sequence(x, mel_fb, hush, weights, shape.n_layer, shape.n_head)
+    return ref, time.perf_counter() - t0
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        n = os.cpu_count() or 1
+    return int(n)
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    shape = I.SHAPES["large"]
+    seed = I.CONFIG_SEED["large"]
+    W = I.encoder_weights(seed, shape)
+    F = I.mel_filterbank(shape.n_mel)
+    hush = I.round_to_bf16(I.hush_mel(seed, shape.n_mel))
+    times = []
+    for it in range(args.warmup + args.steps):
+        _, dt = oracle_sample(W, F, hush, seed)
+        if it >= args.warmup:
+            times.append(dt)
+    mean = sum(times) / len(times)
+    value = SAMPLE_SECONDS / mean
+    sample = (f"stream 0's first {SAMPLE_SECONDS} s + 50 hush frames "
+              f"({int(I.tokens_of([SAMPLE_SECONDS * I.SAMPLE_RATE])[0])} tokens) through all 32 layers, per step")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2412_11272_b200 import build as B
+    from paper_2412_11272_b200.binding import Encoder
+
+    B.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    shape = I.SHAPES["large"]
+    seed = I.CONFIG_SEED["large"]
+    W = I.encoder_weights(seed, shape)
+    F = I.mel_filterbank(shape.n_mel)
+    hush_np = I.round_to_bf16(I.hush_mel(seed, shape.n_mel))
+    hush = torch.as_tensor(hush_np).to(dev)
+
+    # this rank's 64 streams (stream ids continue across ranks: weak scaling, no exchange)
+    streams = np.stack([I.large_stream(seed, rank * N_STREAMS + s) for s in range(N_STREAMS)])
+    max_tokens = int(I.tokens_of([15 * I.SAMPLE_RATE] * N_STREAMS).sum())
+    max_samples = N_STREAMS * 15 * I.SAMPLE_RATE
+    enc = Encoder(shape, W, F, N_STREAMS, max_tokens, max_samples, device=dev)
+    audio_host, audio_dev, lengths = {}, {}, {}
+    for k in ROUNDS:
+        a = np.ascontiguousarray(streams[:, : k * I.SAMPLE_RATE]).reshape(-1)
+        audio_host[k] = torch.as_tensor(a).pin_memory()
+        audio_dev[k] = audio_host[k].to(dev)
+        lengths[k] = np.full(N_STREAMS, k * I.SAMPLE_RATE, dtype=np.int64)
+    out_dev = torch.empty((max_tokens, shape.d_model), dtype=torch.bfloat16, device=dev)
+    out_host = torch.empty((max_tokens, shape.d_model), dtype=torch.bfloat16).pin_memory()
+
+    flops = {k: I.algorithmic_flops(shape, lengths[k]) for k in ROUNDS}
+    step_audio_s = sum(f["audio_seconds"] for f in flops.values())
+    step_tokens = sum(f["tokens"] for f in flops.values())
+    step_flops = sum(f["encoder"] for f in flops.values())
+    step_gemm_flops = sum(f["gemm"] for f in flops.values())
+
+    def step(call_events=None):
+        for k in ROUNDS:
+            if call_events is not None:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+            enc.wf_encode(audio_dev[k], lengths[k], hush, out=out_dev)
+            if call_events is not None:
+                b.record()
+                call_events.append((k, a, b))
+
+    def step_host():
+        for k in ROUNDS:
+            enc.wf_encode_host(audio_host[k], lengths[k], hush, out_host)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if world > 1:
+            t = torch.tensor([x], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return x
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    enc.wf_check()
+
+    sampler = ClockSampler(local_rank)
+    call_events = []
+    enc.wf_profile_enable(True)
+    enc.wf_profile_read()
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step(call_events)
+    e1.record()
+    barrier()
+    clocks = sampler.finish()
+    elapsed_ms = max_over_ranks(e0.elapsed_time(e1))
+    prof = enc.wf_profile_read()
+    enc.wf_profile_enable(False)
+    enc.wf_check()
+
+    # end to end through host buffers: pinned audio in, hidden states out, every call
+    step_host()
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        step_host()
+    t1.record()
+    barrier()
+    e2e_ms = max_over_ranks(t0.elapsed_time(t1))
+
+    if rank != 0:
+        return
+    peaks = measured_peaks()
+    sec = elapsed_ms / 1e3
+    value = world * args.steps * step_audio_s / sec
+    tflops = args.steps * step_flops / sec / 1e12            # per GPU
+    per_buffer = [a.elapsed_time(b) / N_STREAMS for _, a, b in call_events]
+    gemm = prof["block_gemm"]
+    gemm_flops_per_launch = args.steps * step_gemm_flops / max(gemm["launches"], 1)
+    gemm_tflops = gemm_flops_per_launch / (gemm["ms"] / max(gemm["launches"], 1) / 1e3) / 1e12 if gemm["ms"] > 0 else None
+    launches = sum(v["launches"] for v in prof.values()) + prof["front_end"]["launches"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "streams_per_gpu": N_STREAMS, "calls_per_step": len(ROUNDS),
+                   "tokens_per_step": step_tokens, "audio_seconds_per_step": step_audio_s,
+                   "l2": "activations and weights of every call exceed the 126 MB L2 (1.26 GB of weights per call)",
+                   "parallelism": f"dp{world} (independent streams per rank)"},
+        "tokens_per_sec": world * args.steps * step_tokens / sec,
+        "algorithmic_tflops_per_gpu": tflops,
+        "frac_bf16_peak": {"burst": tflops / peaks["bf16_burst"], "sustained": tflops / peaks["bf16_sustained"],
+                           "of": peaks["source"]},
+        "p50_ms_per_buffer": statistics.median(per_buffer), "p90_ms_per_buffer": float(np.percentile(per_buffer, 90)),
+        "clocks": clocks,
+        "e2e": {"value": world * args.steps * step_audio_s / (e2e_ms / 1e3), "unit": UNIT,
+                "h2d_bytes_per_step": int(sum(audio_host[k].numel() * 4 for k in ROUNDS)),
+                "d2h_bytes_per_step": int(step_tokens * shape.d_model * 2)},
+        "gpu_launches": int(launches),
+        "kernel_ms_per_step": {k: v["ms"] / args.steps for k, v in prof.items()},
+        "roofline": {"kernel": "gemm_bf16_kernel (tcgen05, QKV / out-proj / FC1 / FC2)", "bound": "tensor",
+                     "achieved": gemm_tflops, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+                     "frac": (gemm_tflops / peaks["bf16_sustained"]) if gemm_tflops else None,
+                     "peak_kind": f"sustained bf16 matmul, {peaks['source']}",
+                     "frac_of_burst": (gemm_tflops / peaks["bf16_burst"]) if gemm_tflops else None,
+                     "launches": gemm["launches"], "traffic": None},
+    }
+    if world == 1:
+        ref, dt = oracle_sample(W, F, hush_np, seed)
+        k = SAMPLE_SECONDS
+        out, cu = enc.wf_encode(audio_dev[k], lengths[k], hush)
+        got = out[cu[0]:cu[1]].float().cpu().numpy().astype(np.float64)
+        num = (got * ref).sum(axis=1)
+        cos = float(np.min(num / (np.linalg.norm(got, axis=1) * np.linalg.norm(ref, axis=1))))
+        line["parity"] = {"sequence": f"stream 0, {k} s window inside the 64-stream batch",
+                          "max_rel": float(np.max(np.abs(got - ref)) / np.max(np.abs(ref))), "min_token_cosine": cos,
+                          "tolerance": {"max_rel": 3e-2, "cosine": 0.999}}
+        line["cpu_baseline"] = {"value": SAMPLE_SECONDS / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                "sample": f"stream 0's first {SAMPLE_SECONDS} s + 50 hush frames (775 tokens), all 32 layers, {dt:.1f} s of CPU time"}
+    enc.close()
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_ours(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
