@@ -153,6 +153,25 @@ wf_status wf_gemm_bf16(wf_encoder *enc, const void *A, const void *W, const floa
 wf_status wf_attention(wf_encoder *enc, const void *qkv, const int *cu_seqlens, int B, void *out,
                        void *stream);
 
+/* wf_attention_f32_static: wf_attention for float32 activations without an encoder handle and
+ * without any allocation (the paper has no counterpart; this exists for integration only).
+ * It is meant for callers that cannot call cudaMalloc: code running inside a process whose
+ * device memory is owned and fully handed out by another allocator, or a plug-in that is
+ * given pointers and must not grow its host's footprint.  Such callers cannot create an
+ * encoder, because create() allocates workspace.  Here the per-call index arrays (token prefix
+ * sums and query-tile list) live in a fixed 35 KB array inside the library image, held by
+ * every GPU that loads the library until the process exits.
+ *   qkv dev float32 [M, 3 d_model] (q | k | v, head h at columns 64 h), out dev float32
+ *   [M, d_model], cu_seqlens host B+1 strictly increasing from 0; d_model a multiple of 64.
+ * Limits: B <= 256 and M <= 65,536, else WF_ERR_CAPACITY.  No cudaMalloc, cudaFree or other
+ * allocating call is made.  The first call on a device looks up the array's device address
+ * (once per device, with that device current); make that first call outside any stream
+ * capture.  All calls on a device share the array and each overwrites what it reads, so
+ * calls are safe back to back on one stream, but calls that may overlap on the GPU (different
+ * streams without ordering between them) race on it. */
+wf_status wf_attention_f32_static(const float *qkv, const int *cu_seqlens, int B, int d_model,
+                                  float *out, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -54,7 +54,7 @@ _PER_LAYER = ("ln1_g", "ln1_b", "wq", "bq", "wk", "wv", "bv", "wo", "bo", "ln2_g
 
 EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_mel", "wf_encode_host", "wf_check",
            "wf_encoder_destroy", "wf_last_error", "wf_profile_enable", "wf_profile_read",
-           "wf_gemm_bf16", "wf_attention")
+           "wf_gemm_bf16", "wf_attention", "wf_attention_f32_static")
 
 _lib = None
 
@@ -81,6 +81,7 @@ def load_library() -> C.CDLL:
     lib.wf_profile_read.argtypes = [vp, lp, C.POINTER(C.c_double)]
     lib.wf_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, C.c_long, C.c_int, C.c_int, C.c_int, vp]
     lib.wf_attention.argtypes = [vp, vp, ip, C.c_int, vp, vp]
+    lib.wf_attention_f32_static.argtypes = [vp, ip, C.c_int, C.c_int, vp, vp]
     for name in EXPORTS:
         if name != "wf_last_error":
             getattr(lib, name).restype = C.c_int
@@ -248,3 +249,15 @@ class Encoder:
         self._check(self.lib.wf_attention(self.handle, qkv.data_ptr(), cu.ctypes.data_as(C.POINTER(C.c_int)),
                                           len(cu) - 1, out.data_ptr(), _stream_ptr(stream)))
         return out
+
+
+def wf_attention_f32_static(qkv: torch.Tensor, cu_seqlens, d_model: int, out: torch.Tensor, stream=None):
+    """Handle-free float32 attention that makes no allocation of its own: the caller passes the
+    output tensor too.  For code that may not call cudaMalloc (see the header).  Raises WfError."""
+    lib = load_library()
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+    st = lib.wf_attention_f32_static(qkv.data_ptr(), cu.ctypes.data_as(C.POINTER(C.c_int)), len(cu) - 1,
+                                     int(d_model), out.data_ptr(), _stream_ptr(stream))
+    if st != 0:
+        raise WfError(st, "wf_attention_f32_static rejected its arguments or a CUDA call failed")
+    return out
