@@ -44,6 +44,7 @@ struct wf_encoder {
   float *conv1_b, *conv2_b, *lnp_g, *lnp_b;
   std::vector<LayerW> layers;
   CUtensorMap tm_conv1_w, tm_conv2_w, tm_zp, tm_c1p, tm_h, tm_attn, tm_fc1;
+  CUtensorMap tmo_c1p, tmo_qkv, tmo_fc1, tmo_x;  // epilogue outputs
 
   float* logmel;
   int* seq_max;
@@ -255,9 +256,10 @@ wf_status ring_release(wf_encoder* e, int slot, cudaStream_t s) {
   return WF_OK;
 }
 
-void gemm(wf_encoder* e, const CUtensorMap* ta, const CUtensorMap* tb, const void* A, long lda, const void* W,
-          long ldw, long M, int N, int K, int a_cols, int epi, const EpiParams& ep, cudaStream_t s) {
-  if (e->bf16) launch_gemm_bf16(*ta, *tb, M, N, K, a_cols, epi, ep, e->err_flag, e->num_sms, s);
+void gemm(wf_encoder* e, const CUtensorMap* ta, const CUtensorMap* tb, const CUtensorMap* tc, const void* A,
+          long lda, const void* W, long ldw, long M, int N, int K, int a_cols, int epi, const EpiParams& ep,
+          cudaStream_t s) {
+  if (e->bf16) launch_gemm_bf16(*ta, *tb, *tc, M, N, K, a_cols, epi, ep, e->err_flag, e->num_sms, s);
   else launch_gemm_f32((const float*)A, lda, (const float*)W, ldw, M, N, K, epi, ep, s);
 }
 
@@ -275,14 +277,14 @@ wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidde
     Prof pr(e, 2, s);
     EpiParams ep{};
     ep.bias = e->conv1_b; ep.out = e->c1p; ep.ldc = d; ep.row_valid = e->row_valid;
-    gemm(e, &e->tm_zp, &e->tm_conv1_w, e->zp_alloc, e->mel_ld, e->conv1_w, 3L * e->mel_ld, p.total_prows, d,
+    gemm(e, &e->tm_zp, &e->tm_conv1_w, &e->tmo_c1p, e->zp_alloc, e->mel_ld, e->conv1_w, 3L * e->mel_ld, p.total_prows, d,
          3 * e->mel_ld, e->mel_ld, kEpiConv1, ep, s);
   }
   {
     Prof pr(e, 2, s);
     EpiParams ep{};
     ep.bias = e->conv2_b; ep.resid = e->x; ep.ldc = d; ep.row_dst = e->row_dst; ep.pe = e->pe;
-    gemm(e, &e->tm_c1p, &e->tm_conv2_w, e->c1p, 2L * d, e->conv2_w, 3L * d, p.total_prows / 2, d, 3 * d, 2 * d,
+    gemm(e, &e->tm_c1p, &e->tm_conv2_w, &e->tmo_x, e->c1p, 2L * d, e->conv2_w, 3L * d, p.total_prows / 2, d, 3 * d, 2 * d,
          kEpiConv2, ep, s);
   }
   for (int l = 0; l < c.n_layer; ++l) {
@@ -295,7 +297,7 @@ wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidde
       Prof pr(e, 4, s);
       EpiParams ep{};
       ep.bias = w.bqkv; ep.out = e->qkv; ep.ldc = 3L * d;
-      gemm(e, &e->tm_h, &w.tm_wqkv, e->h, d, w.wqkv, d, M, 3 * d, d, d, kEpiBias, ep, s);
+      gemm(e, &e->tm_h, &w.tm_wqkv, &e->tmo_qkv, e->h, d, w.wqkv, d, M, 3 * d, d, d, kEpiBias, ep, s);
     }
     {
       Prof pr(e, 5, s);
@@ -306,7 +308,7 @@ wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidde
       Prof pr(e, 4, s);
       EpiParams ep{};
       ep.bias = w.bo; ep.resid = e->x; ep.ldc = d;
-      gemm(e, &e->tm_attn, &w.tm_wo, e->attn, d, w.wo, d, M, d, d, d, kEpiBiasResid, ep, s);
+      gemm(e, &e->tm_attn, &w.tm_wo, &e->tmo_x, e->attn, d, w.wo, d, M, d, d, d, kEpiBiasResid, ep, s);
     }
     {
       Prof pr(e, 3, s);
@@ -316,13 +318,13 @@ wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidde
       Prof pr(e, 4, s);
       EpiParams ep{};
       ep.bias = w.b1; ep.out = e->fc1; ep.ldc = F;
-      gemm(e, &e->tm_h, &w.tm_w1, e->h, d, w.w1, d, M, F, d, d, kEpiBiasGelu, ep, s);
+      gemm(e, &e->tm_h, &w.tm_w1, &e->tmo_fc1, e->h, d, w.w1, d, M, F, d, d, kEpiBiasGelu, ep, s);
     }
     {
       Prof pr(e, 4, s);
       EpiParams ep{};
       ep.bias = w.b2; ep.resid = e->x; ep.ldc = d;
-      gemm(e, &e->tm_fc1, &w.tm_w2, e->fc1, F, w.w2, F, M, d, F, F, kEpiBiasResid, ep, s);
+      gemm(e, &e->tm_fc1, &w.tm_w2, &e->tmo_x, e->fc1, F, w.w2, F, M, d, F, F, kEpiBiasResid, ep, s);
     }
   }
   {
@@ -497,6 +499,10 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     ok &= make_tmap_bf16(e->tma, &e->tm_h, e->h, d, mt, d, 128);
     ok &= make_tmap_bf16(e->tma, &e->tm_attn, e->attn, d, mt, d, 128);
     ok &= make_tmap_bf16(e->tma, &e->tm_fc1, e->fc1, F, mt, F, 128);
+    ok &= make_tmap_out(e->tma, &e->tmo_c1p, e->c1p, 2, d, e->cap_prows + 4);
+    ok &= make_tmap_out(e->tma, &e->tmo_qkv, e->qkv, 2, 3 * d, mt);
+    ok &= make_tmap_out(e->tma, &e->tmo_fc1, e->fc1, 2, F, mt);
+    ok &= make_tmap_out(e->tma, &e->tmo_x, e->x, 4, d, mt);
     ok &= make_tmap_bf16(e->tma, &e->tm_conv1_w, e->conv1_w, 3 * e->mel_ld, d, 3 * e->mel_ld, 256);
     ok &= make_tmap_bf16(e->tma, &e->tm_conv2_w, e->conv2_w, 3 * d, d, 3 * d, 256);
     for (int l = 0; l < c.n_layer; ++l) {
@@ -645,14 +651,15 @@ wf_status wf_gemm_bf16(wf_encoder* e, const void* A, const void* W, const float*
       ((uintptr_t)A & 15) || ((uintptr_t)W & 15) || ((uintptr_t)C & 15) || ((uintptr_t)bias & 15))
     return fail(e, WF_ERR_INVALID_ARG, "wf_gemm_bf16: bad pointer, size or mode");
   if (M == 0) return WF_OK;
-  CUtensorMap ta, tb;
-  if (!make_tmap_bf16(e->tma, &ta, A, K, M, K, 128) || !make_tmap_bf16(e->tma, &tb, W, K, N, K, 256))
+  CUtensorMap ta, tb, tc;
+  if (!make_tmap_bf16(e->tma, &ta, A, K, M, K, 128) || !make_tmap_bf16(e->tma, &tb, W, K, N, K, 256) ||
+      !make_tmap_out(e->tma, &tc, C, mode == 2 ? 4 : 2, N, M))
     return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
   EpiParams ep{};
   ep.bias = bias;
   ep.ldc = N;
   if (mode == 2) ep.resid = (float*)C; else ep.out = C;
-  launch_gemm_bf16(ta, tb, M, N, K, K, mode, ep, e->err_flag, e->num_sms, (cudaStream_t)stream);
+  launch_gemm_bf16(ta, tb, tc, M, N, K, K, mode, ep, e->err_flag, e->num_sms, (cudaStream_t)stream);
   WF_CUDA(e, cudaGetLastError());
   return WF_OK;
 }

@@ -5,8 +5,11 @@
 //               into a ring of shared-memory stages guarded by full/empty mbarriers;
 //   warp 1      allocates tensor memory, one lane issues tcgen05.mma (128 x BN x 16, f32
 //               accumulation in TMEM) and commits stage releases / accumulator readiness;
-//   warps 2..5  read the accumulator with tcgen05.ld (one row per thread) and apply the fused
-//               epilogue while the MMA warp already fills the other accumulator buffer.
+//   warps 2..5  read the accumulator with tcgen05.ld (one row per thread), apply the fused
+//               epilogue, stage 32-row x 128-byte pieces in swizzled shared memory and hand them
+//               to TMA: a tile store for bf16 outputs, a float32 add-reduction (performed at the
+//               L2) for the residual update, so the residual is never read by the SM.  This runs
+//               while the MMA warp already fills the other accumulator buffer.
 // Every mbarrier wait is bounded; on a timeout the CTA sets an error word, drains its own
 // TMA copies, frees its tensor memory and returns.
 #include "wf_internal.h"
@@ -27,79 +30,54 @@ struct GemmCfg {
   static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = BN * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kBarOffset = kStages * kStageBytes;
+  static constexpr int kStagingOffset = kStages * kStageBytes;       // 4 warps x 2 buffers x 4 KB
+  static constexpr int kStagingBytes = 4 * 2 * 4096;
+  static constexpr int kBarOffset = kStagingOffset + kStagingBytes;
   static constexpr int kSmemBytes = kBarOffset + 256 + 1024;  // barriers + alignment slack
   static constexpr int kTmemCols = 2 * BN;
 };
 
-// One accumulator row segment: 32 consecutive columns starting at col0 for GEMM row `row`.
+// bias add (+ GELU) of 32 accumulator columns starting at col0 (col0 + 32 <= padded N is not
+// required: columns at or beyond N are computed from a clamped bias index and never stored).
 template <int EPI>
-__device__ __forceinline__ void epilogue_row32(const EpiParams& ep, long row, long M, int col0, int N,
-                                               const uint32_t (&acc)[32]) {
-  if (row >= M || col0 >= N) return;
-  long orow = row;
-  bool valid = true;
-  int pos = 0;
-  if (EPI == kEpiConv1) valid = ep.row_valid[row] != 0;
-  if (EPI == kEpiConv2) {
-    int2 d = ep.row_dst[row];
-    if (d.x < 0) return;
-    orow = d.x;
-    pos = d.y;
+__device__ __forceinline__ void bias_act32(const EpiParams& ep, int col0, int N, const uint32_t (&acc)[32],
+                                           float (&v)[32]) {
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    int col = col0 + 4 * g;
+    float4 b = col < N ? __ldg(reinterpret_cast<const float4*>(ep.bias + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    v[4 * g + 0] = __uint_as_float(acc[4 * g + 0]) + b.x;
+    v[4 * g + 1] = __uint_as_float(acc[4 * g + 1]) + b.y;
+    v[4 * g + 2] = __uint_as_float(acc[4 * g + 2]) + b.z;
+    v[4 * g + 3] = __uint_as_float(acc[4 * g + 3]) + b.w;
   }
+  if (EPI == kEpiBiasGelu || EPI == kEpiConv1 || EPI == kEpiConv2) {
 #pragma unroll
-  for (int g = 0; g < 4; ++g) {  // groups of 8 columns
-    int col = col0 + 8 * g;
+    for (int i = 0; i < 32; ++i) v[i] = gelu_sigmoid_poly(v[i]);
+  }
+}
+
+// Direct (non-TMA) store of one row segment for the stride-2 conv epilogue, whose output rows
+// are remapped per sequence: resid[dst] = gelu(acc + bias) + pe[pos].
+__device__ __forceinline__ void conv2_store32(const EpiParams& ep, long row, long M, int col0, int N,
+                                              const float (&v)[32]) {
+  if (row >= M || col0 >= N) return;
+  int2 d = ep.row_dst[row];
+  if (d.x < 0) return;
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    int col = col0 + 4 * g;
     if (col >= N) break;
-    float v[8];
-    float4 b0 = __ldg(reinterpret_cast<const float4*>(ep.bias + col));
-    float4 b1 = __ldg(reinterpret_cast<const float4*>(ep.bias + col + 4));
-    v[0] = __uint_as_float(acc[8 * g + 0]) + b0.x;
-    v[1] = __uint_as_float(acc[8 * g + 1]) + b0.y;
-    v[2] = __uint_as_float(acc[8 * g + 2]) + b0.z;
-    v[3] = __uint_as_float(acc[8 * g + 3]) + b0.w;
-    v[4] = __uint_as_float(acc[8 * g + 4]) + b1.x;
-    v[5] = __uint_as_float(acc[8 * g + 5]) + b1.y;
-    v[6] = __uint_as_float(acc[8 * g + 6]) + b1.z;
-    v[7] = __uint_as_float(acc[8 * g + 7]) + b1.w;
-    if (EPI == kEpiBiasGelu || EPI == kEpiConv1 || EPI == kEpiConv2) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) v[i] = gelu_erf(v[i]);
-    }
-    if (EPI == kEpiBias || EPI == kEpiBiasGelu || EPI == kEpiConv1) {
-      if (EPI == kEpiConv1 && !valid) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = 0.f;
-      }
-      __nv_bfloat162 p0 = __floats2bfloat162_rn(v[0], v[1]), p1 = __floats2bfloat162_rn(v[2], v[3]);
-      __nv_bfloat162 p2 = __floats2bfloat162_rn(v[4], v[5]), p3 = __floats2bfloat162_rn(v[6], v[7]);
-      uint4 u;
-      u.x = *reinterpret_cast<uint32_t*>(&p0);
-      u.y = *reinterpret_cast<uint32_t*>(&p1);
-      u.z = *reinterpret_cast<uint32_t*>(&p2);
-      u.w = *reinterpret_cast<uint32_t*>(&p3);
-      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.out) + orow * ep.ldc + col) = u;
-    } else if (EPI == kEpiBiasResid) {
-      float4* p = reinterpret_cast<float4*>(ep.resid + orow * ep.ldc + col);
-      float4 r0 = p[0], r1 = p[1];
-      r0.x += v[0]; r0.y += v[1]; r0.z += v[2]; r0.w += v[3];
-      r1.x += v[4]; r1.y += v[5]; r1.z += v[6]; r1.w += v[7];
-      p[0] = r0;
-      p[1] = r1;
-    } else {  // kEpiConv2
-      const float4* pe = reinterpret_cast<const float4*>(ep.pe + (long)pos * ep.ldc + col);
-      float4 e0 = __ldg(pe), e1 = __ldg(pe + 1);
-      float4* p = reinterpret_cast<float4*>(ep.resid + orow * ep.ldc + col);
-      p[0] = make_float4(v[0] + e0.x, v[1] + e0.y, v[2] + e0.z, v[3] + e0.w);
-      p[1] = make_float4(v[4] + e1.x, v[5] + e1.y, v[6] + e1.z, v[7] + e1.w);
-    }
+    float4 e = __ldg(reinterpret_cast<const float4*>(ep.pe + (long)d.y * ep.ldc + col));
+    *reinterpret_cast<float4*>(ep.resid + (long)d.x * ep.ldc + col) =
+        make_float4(v[4 * g] + e.x, v[4 * g + 1] + e.y, v[4 * g + 2] + e.z, v[4 * g + 3] + e.w);
   }
 }
 
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
-    const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, long M, int N,
-    int K, int a_cols, EpiParams ep, int* err_flag) {
+    const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+    const __grid_constant__ CUtensorMap tmap_c, long M, int N, int K, int a_cols, EpiParams ep, int* err_flag) {
   using Cfg = GemmCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -210,6 +188,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
     }
   } else {
     const int quarter = warp & 3;  // TMEM lanes this warp may read: 32 * quarter .. + 31
+    const uint32_t stage_base = smem_base + Cfg::kStagingOffset + (uint32_t)((warp - 2) * 8192);
+    uint32_t piece = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
@@ -223,18 +203,86 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
       tc_fence_after();
       const long row = (long)m0 + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+      if (EPI == kEpiConv2) {
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld_32x32(t_row + c * 32, v);
-        tmem_ld_wait();
-        epilogue_row32<EPI>(ep, row, M, n0 + c * 32, N, v);
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t a32[32];
+          float v[32];
+          tmem_ld_32x32(t_row + c * 32, a32);
+          tmem_ld_wait();
+          bias_act32<EPI>(ep, n0 + c * 32, N, a32, v);
+          conv2_store32(ep, row, M, n0 + c * 32, N, v);
+        }
+      } else if (EPI == kEpiBiasResid) {
+        // float32: 32 columns = 128 bytes per row and piece
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          const uint32_t buf = stage_base + (uint32_t)((piece & 1) * 4096);
+          if (lane == 0) bulk_wait_read<1>();   // the copy that last read this buffer is done with it
+          __syncwarp();
+          uint32_t a32[32];
+          float v[32];
+          tmem_ld_32x32(t_row + c * 32, a32);
+          tmem_ld_wait();
+          bias_act32<EPI>(ep, n0 + c * 32, N, a32, v);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(buf + lane * 128 + ((j ^ (lane & 7)) << 4), __float_as_uint(v[4 * j]),
+                         __float_as_uint(v[4 * j + 1]), __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0 && n0 + c * 32 < N && (long)m0 + quarter * 32 < M) {
+            tma_reduce_add_2d(&tmap_c, buf, n0 + c * 32, m0 + quarter * 32);
+            bulk_commit();
+          }
+          ++piece;
+        }
+      } else {
+        // bf16: 64 columns = 128 bytes per row and piece
+        bool valid = true;
+        if (EPI == kEpiConv1) valid = row < M && ep.row_valid[row] != 0;
+#pragma unroll 1
+        for (int c = 0; c < BN / 64; ++c) {
+          const uint32_t buf = stage_base + (uint32_t)((piece & 1) * 4096);
+          if (lane == 0) bulk_wait_read<1>();
+          __syncwarp();
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            uint32_t a32[32];
+            float v[32];
+            tmem_ld_32x32(t_row + c * 64 + hf * 32, a32);
+            tmem_ld_wait();
+            bias_act32<EPI>(ep, n0 + c * 64 + hf * 32, N, a32, v);
+            if (EPI == kEpiConv1 && !valid) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) v[i] = 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              __nv_bfloat162 p0 = __floats2bfloat162_rn(v[8 * j + 0], v[8 * j + 1]);
+              __nv_bfloat162 p1 = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
+              __nv_bfloat162 p2 = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
+              __nv_bfloat162 p3 = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
+              st_shared_v4(buf + lane * 128 + (((hf * 4 + j) ^ (lane & 7)) << 4), *reinterpret_cast<uint32_t*>(&p0),
+                           *reinterpret_cast<uint32_t*>(&p1), *reinterpret_cast<uint32_t*>(&p2),
+                           *reinterpret_cast<uint32_t*>(&p3));
+            }
+          }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0 && n0 + c * 64 < N && (long)m0 + quarter * 32 < M) {
+            tma_store_2d(&tmap_c, buf, n0 + c * 64, m0 + quarter * 32);
+            bulk_commit();
+          }
+          ++piece;
+        }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    if (lane == 0) bulk_wait_all();  // every store / reduction this lane issued has completed
   }
 
   tc_fence_before();
@@ -260,17 +308,27 @@ bool tma_api_init(TmaApi* api) {
   return true;
 }
 
-bool make_tmap_bf16(const TmaApi& api, CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows,
-                    uint64_t pitch_elems, uint32_t box_rows) {
+bool make_tmap_2d(const TmaApi& api, CUtensorMap* m, const void* base, int elem_bytes, uint64_t cols,
+                  uint64_t rows, uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows) {
   cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {pitch_elems * 2};
-  cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+  cuuint64_t strides[1] = {pitch_elems * (uint64_t)elem_bytes};
+  cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = reinterpret_cast<EncodeTiledFn>(api.encode_tiled)(
-      m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      m, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+      const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+
+bool make_tmap_bf16(const TmaApi& api, CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows,
+                    uint64_t pitch_elems, uint32_t box_rows) {
+  return make_tmap_2d(api, m, base, 2, cols, rows, pitch_elems, (uint32_t)kBK, box_rows);
+}
+
+bool make_tmap_out(const TmaApi& api, CUtensorMap* m, const void* base, int elem_bytes, uint64_t cols,
+                   uint64_t rows) {
+  return make_tmap_2d(api, m, base, elem_bytes, cols, rows, cols, elem_bytes == 2 ? 64 : 32, 32);
 }
 
 template <int BN, int EPI>
@@ -290,23 +348,23 @@ cudaError_t gemm_bf16_configure() {
 }
 
 template <int BN, int EPI>
-static void launch_one(const CUtensorMap& ta, const CUtensorMap& tb, long M, int N, int K, int a_cols,
-                       const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
+static void launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
+                       int a_cols, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
   const long tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
   const int grid = (int)(tiles < num_sms ? tiles : num_sms);
-  gemm_bf16_kernel<BN, EPI><<<grid, kGemmThreads, GemmCfg<BN>::kSmemBytes, s>>>(ta, tb, M, N, K, a_cols, ep,
+  gemm_bf16_kernel<BN, EPI><<<grid, kGemmThreads, GemmCfg<BN>::kSmemBytes, s>>>(ta, tb, tc, M, N, K, a_cols, ep,
                                                                                  err_flag);
 }
 
-void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, long M, int N, int K, int a_cols,
-                      int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
+void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
+                      int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
   if (M <= 0 || N <= 0 || K <= 0) return;
   switch (epi) {
-    case kEpiBias: launch_one<256, kEpiBias>(ta, tb, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-    case kEpiBiasGelu: launch_one<256, kEpiBiasGelu>(ta, tb, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-    case kEpiBiasResid: launch_one<256, kEpiBiasResid>(ta, tb, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-    case kEpiConv1: launch_one<256, kEpiConv1>(ta, tb, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-    default: launch_one<256, kEpiConv2>(ta, tb, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    case kEpiBias: launch_one<256, kEpiBias>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    case kEpiBiasGelu: launch_one<256, kEpiBiasGelu>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    case kEpiBiasResid: launch_one<256, kEpiBiasResid>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    case kEpiConv1: launch_one<256, kEpiConv1>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    default: launch_one<256, kEpiConv2>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
   }
 }
 

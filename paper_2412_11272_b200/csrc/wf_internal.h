@@ -87,11 +87,17 @@ bool tma_api_init(TmaApi* api);
 // elements, box = 64 x box_rows, 128 B swizzle.
 bool make_tmap_bf16(const TmaApi& api, CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows,
                     uint64_t pitch_elems, uint32_t box_rows);
+// Output tensor map for the epilogue's TMA stores: box of 32 rows x 128 bytes (64 bf16 or 32 f32).
+bool make_tmap_out(const TmaApi& api, CUtensorMap* m, const void* base, int elem_bytes, uint64_t cols,
+                   uint64_t rows);
 cudaError_t gemm_bf16_configure();
 // a_cols: stored row length of A in elements (K for a plain GEMM; smaller when one GEMM row
 // spans several consecutive stored rows, which must then be a multiple of 64).
-void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, long M, int N, int K, int a_cols,
-                      int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s);
+// tc: output map (bf16 out for kEpiBias/kEpiBiasGelu/kEpiConv1, float32 residual for
+// kEpiBiasResid; unused by kEpiConv2).  Rows of the output between M and the next multiple of
+// 128 are written too when the map has them: outputs must be capacity-sized or exactly M rows.
+void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
+                      int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s);
 
 // ---- bf16 attention (wf_attention.cu)
 cudaError_t attention_bf16_configure();
