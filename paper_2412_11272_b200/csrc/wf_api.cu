@@ -45,6 +45,7 @@ struct wf_encoder {
   std::vector<LayerW> layers;
   CUtensorMap tm_conv1_w, tm_conv2_w, tm_zp, tm_c1p, tm_h, tm_attn, tm_fc1;
   CUtensorMap tmo_c1p, tmo_qkv, tmo_fc1, tmo_x;  // epilogue outputs
+  CUtensorMap tm_qkv, tm_qkv_kv;                 // attention operand loads (128- and 64-row boxes)
 
   float* logmel;
   int* seq_max;
@@ -208,7 +209,7 @@ wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Pl
   hm[ml.tok_off + B] = (int)tokens;
   hm[ml.fe_tile_off + B] = (int)tiles;
   // attention work list: (sequence, first query row), longest sequences first
-  const int qt = e->bf16 ? 64 : 16;
+  const int qt = e->bf16 ? 256 : 16;
   std::vector<int> order(B);
   for (int i = 0; i < B; ++i) order[i] = i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
@@ -301,7 +302,7 @@ wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidde
     }
     {
       Prof pr(e, 5, s);
-      if (e->bf16) launch_attention_bf16((const __nv_bfloat16*)e->qkv, (__nv_bfloat16*)e->attn, meta, p.ml, p.n_work, d, s);
+      if (e->bf16) launch_attention_bf16(e->tm_qkv, e->tm_qkv_kv, (__nv_bfloat16*)e->attn, meta, p.ml, p.n_work, d, e->err_flag, e->num_sms, s);
       else launch_attention_f32((const float*)e->qkv, (float*)e->attn, meta, p.ml, p.n_work, d, s);
     }
     {
@@ -499,6 +500,8 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     ok &= make_tmap_bf16(e->tma, &e->tm_h, e->h, d, mt, d, 128);
     ok &= make_tmap_bf16(e->tma, &e->tm_attn, e->attn, d, mt, d, 128);
     ok &= make_tmap_bf16(e->tma, &e->tm_fc1, e->fc1, F, mt, F, 128);
+    ok &= make_tmap_bf16(e->tma, &e->tm_qkv, e->qkv, 3 * d, mt, 3 * d, 128);
+    ok &= make_tmap_bf16(e->tma, &e->tm_qkv_kv, e->qkv, 3 * d, mt, 3 * d, 64);
     ok &= make_tmap_out(e->tma, &e->tmo_c1p, e->c1p, 2, d, e->cap_prows + 4);
     ok &= make_tmap_out(e->tma, &e->tmo_qkv, e->qkv, 2, 3 * d, mt);
     ok &= make_tmap_out(e->tma, &e->tmo_fc1, e->fc1, 2, F, mt);
@@ -618,7 +621,7 @@ wf_status wf_check(wf_encoder* e, void* stream) {
   WF_CUDA(e, cudaMemcpy(&flag, e->err_flag, sizeof(int), cudaMemcpyDeviceToHost));
   if (flag != 0) {
     cudaMemset(e->err_flag, 0, sizeof(int));
-    return fail(e, WF_ERR_DEVICE_TIMEOUT, "a bounded wait inside a GEMM kernel gave up (role %d)", flag);
+    return fail(e, WF_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel gave up (role code %d: 1-3 GEMM, 11-13 attention)", flag);
   }
   return WF_OK;
 }
@@ -682,7 +685,7 @@ wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, in
   ml.tok_off = 0;
   ml.attn_work = B + 1;
   for (int i = 0; i <= B; ++i) hm[i] = cu_seqlens[i];
-  const int qt = e->bf16 ? 64 : 16;
+  const int qt = e->bf16 ? 256 : 16;
   int nw = 0;
   for (int i = 0; i < B; ++i)
     for (int q0 = 0; q0 < cu_seqlens[i + 1] - cu_seqlens[i]; q0 += qt) {
@@ -697,7 +700,13 @@ wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, in
   if (st != WF_OK) return st;
   {
     Prof pr(e, 5, s);
-    if (e->bf16) launch_attention_bf16((const __nv_bfloat16*)qkv, (__nv_bfloat16*)out, e->meta_dev[slot], ml, nw, e->cfg.d_model, s);
+    if (e->bf16) {
+      CUtensorMap tq, tkv;
+      if (!make_tmap_bf16(e->tma, &tq, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 128) ||
+          !make_tmap_bf16(e->tma, &tkv, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 64))
+        return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected the qkv tensor map");
+      launch_attention_bf16(tq, tkv, (__nv_bfloat16*)out, e->meta_dev[slot], ml, nw, e->cfg.d_model, e->err_flag, e->num_sms, s);
+    }
     else launch_attention_f32((const float*)qkv, (float*)out, e->meta_dev[slot], ml, nw, e->cfg.d_model, s);
   }
   WF_CUDA(e, cudaGetLastError());

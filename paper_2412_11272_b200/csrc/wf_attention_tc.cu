@@ -1,0 +1,410 @@
+// Non-causal variable-length attention on the 5th-generation tensor cores (bf16, head dim 64).
+//
+// A persistent CTA (352 threads) walks a list of work items; one item = up to 256 query rows
+// (two tiles of 128) of one (sequence, head); keys are consumed 64 at a time.  Roles:
+//   warps 0-3 / 4-7  softmax for query tile 0 / 1, one thread per query row.  A step loads the
+//                    64 scores of its row from tensor memory once, releases the score buffer,
+//                    takes the row maximum, exponentiates, writes the probabilities back to
+//                    tensor memory as packed bf16 (double-buffered) and only then folds in the
+//                    P V product of the PREVIOUS step, so it never waits on the tensor pipe in
+//                    steady state.  The running output row lives in registers.
+//   warp 8           one lane issues the TMA loads: Q tiles once per item, K and V tiles of 64
+//                    keys through two 4-stage rings.
+//   warps 9, 10      MMA issue for query tile 0 / 1 (warp 9 also owns the tensor-memory
+//                    allocation).  The whole warp runs the loop so that descriptors stay in
+//                    uniform registers; one elected lane issues S = Q K^T (128x64x64, operands in
+//                    shared memory) as soon as the softmax has read the previous scores, and
+//                    O = P V (128x64x64, P from tensor memory, V from shared memory as an MN-major
+//                    operand) when the probabilities are in place.  A K / V stage is released
+//                    when both tiles' MMAs on it have completed (barriers count two arrivals).
+// Keys are addressed through the token prefix sums: a key tile that runs past the end of its
+// sequence is masked in the softmax, so no padded token ever contributes.
+// Tensor-memory columns per query tile t (base 256 t): S [0,64) f32; P0 [64,96), P1 [96,128)
+// packed bf16; O0 [128,192), O1 [192,256) f32.  Every mbarrier wait is bounded (wf_ptx.cuh).
+#include "wf_internal.h"
+#include "wf_ptx.cuh"
+
+namespace wf {
+
+using namespace ptx;
+
+namespace {
+
+constexpr int kTQ = 128;          // query rows per tile
+constexpr int kTK = 64;           // keys per step
+constexpr int kKvStages = 4;
+constexpr int kQBytes = kTQ * 64 * 2;      // 16 KB
+constexpr int kKvBytes = kTK * 64 * 2;     // 8 KB
+constexpr int kAttnThreads = 352;
+
+// shared-memory map (offsets from a 1024-byte aligned base)
+constexpr int kOffQ = 0;                                   // 2 tiles
+constexpr int kOffK = kOffQ + 2 * kQBytes;
+constexpr int kOffV = kOffK + kKvStages * kKvBytes;
+constexpr int kOffBar = kOffV + kKvStages * kKvBytes;
+// q_full, q_free | k_full, k_free, v_full, v_free per stage | per tile: s_full, s_free, p_full[2], o_full[2]
+constexpr int kNumBars = 2 + 4 * kKvStages + 2 * 6;
+constexpr int kAttnSmem = kOffBar + 8 * kNumBars + 16 + 1024;
+
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr) {
+  // rows are the K index (a key), the 64 contiguous elements of a row are the N index:
+  // 8-row groups are 1024 B apart (stride byte offset); there is a single 64-wide N block.
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+struct Item {
+  int tok0, n, q0, head, n_kv;
+  bool two;
+};
+
+__device__ __forceinline__ Item load_item(const int* __restrict__ meta, const MetaLayout& ml, int it, int n_head) {
+  Item w;
+  const int work = it / n_head;
+  w.head = it - work * n_head;
+  const int seq = meta[ml.attn_work + 2 * work];
+  w.q0 = meta[ml.attn_work + 2 * work + 1];
+  w.tok0 = meta[ml.tok_off + seq];
+  w.n = meta[ml.tok_off + seq + 1] - w.tok0;
+  w.n_kv = (w.n + kTK - 1) / kTK;
+  w.two = w.q0 + kTQ < w.n;
+  return w;
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
+    const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
+    __nv_bfloat16* __restrict__ out, const int* __restrict__ meta, MetaLayout ml, int n_items, int n_head,
+    int d_model, int* err_flag) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
+  const uint32_t bars = sbase + kOffBar;
+  const uint32_t q_full = bars, q_free = bars + 8;
+  auto k_full = [&](int s) { return bars + 8u * (2 + s); };
+  auto k_free = [&](int s) { return bars + 8u * (2 + kKvStages + s); };
+  auto v_full = [&](int s) { return bars + 8u * (2 + 2 * kKvStages + s); };
+  auto v_free = [&](int s) { return bars + 8u * (2 + 3 * kKvStages + s); };
+  const uint32_t tile_bars = bars + 8u * (2 + 4 * kKvStages);
+  auto s_full = [&](int t) { return tile_bars + 8u * (6 * t); };
+  auto s_free = [&](int t) { return tile_bars + 8u * (6 * t + 1); };
+  auto p_full = [&](int t, int b) { return tile_bars + 8u * (6 * t + 2 + b); };
+  auto o_full = [&](int t, int b) { return tile_bars + 8u * (6 * t + 4 + b); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sgen + kOffBar + 8 * kNumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + kOffBar + 8 * kNumBars + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    mbar_init(q_free, 2);
+    for (int s = 0; s < kKvStages; ++s) {
+      mbar_init(k_full(s), 1);
+      mbar_init(k_free(s), 2);
+      mbar_init(v_full(s), 1);
+      mbar_init(v_free(s), 2);
+    }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(s_full(t), 1);
+      mbar_init(s_free(t), 128);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(p_full(t, b), 128);
+        mbar_init(o_full(t, b), 1);
+      }
+    }
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 9) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 8) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      prefetch_tmap(&tmap_q);
+      prefetch_tmap(&tmap_kv);
+      uint32_t kc = 0, vc = 0, items = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
+        const Item w = load_item(meta, ml, it, n_head);
+        if (!mbar_wait(q_free, (items & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        mbar_arrive_expect_tx(q_full, w.two ? 2 * kQBytes : kQBytes);
+        tma_load_2d(sbase + kOffQ, &tmap_q, w.head * kHeadDim, w.tok0 + w.q0, q_full);
+        if (w.two) tma_load_2d(sbase + kOffQ + kQBytes, &tmap_q, w.head * kHeadDim, w.tok0 + w.q0 + kTQ, q_full);
+        for (int j = 0; j < w.n_kv; ++j) {
+          int s = kc % kKvStages;
+          if (!mbar_wait(k_free(s), ((kc / kKvStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_arrive_expect_tx(k_full(s), kKvBytes);
+          tma_load_2d(sbase + kOffK + s * kKvBytes, &tmap_kv, d_model + w.head * kHeadDim, w.tok0 + j * kTK, k_full(s));
+          ++kc;
+          s = vc % kKvStages;
+          if (!mbar_wait(v_free(s), ((vc / kKvStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_arrive_expect_tx(v_full(s), kKvBytes);
+          tma_load_2d(sbase + kOffV + s * kKvBytes, &tmap_kv, 2 * d_model + w.head * kHeadDim, w.tok0 + j * kTK, v_full(s));
+          ++vc;
+        }
+        ++items;
+      }
+      if (!ok) {
+        atomicExch(err_flag, 11);
+        // bounded drain: give the copies already issued time to land
+        for (uint32_t it2 = 0; it2 < (1u << 16); ++it2) {
+          bool all = mbar_try_wait(q_full, (items & 1u));
+          for (int s = 0; s < kKvStages; ++s) all = all && mbar_try_wait(k_full(s), 0) && mbar_try_wait(v_full(s), 0);
+          if (all) break;
+        }
+      }
+    }
+  } else if (warp == 9 || warp == 10) {
+    // ------------------------------------------------------------------ MMA issue for tile t
+    const int t = warp - 9;
+    constexpr uint32_t idesc_s = umma_idesc_bf16(kTQ, kTK, 0, 0);
+    constexpr uint32_t idesc_o = umma_idesc_bf16(kTQ, kHeadDim, 0, 1);
+    const bool leader = elect_one();
+    const uint64_t qd = umma_desc_k_sw128(sbase + kOffQ + t * kQBytes);
+    const uint64_t kd0 = umma_desc_k_sw128(sbase + kOffK);
+    const uint64_t vd0 = umma_desc_mn_sw128(sbase + kOffV);
+    const uint32_t tm_s = tmem_base + t * 256;
+    uint32_t kc = 0, vc = 0, items = 0, g = 0;  // g: steps done; buffer = g & 1, parity = (g >> 1) & 1
+    bool ok = true;
+    // every lane waits; the verdict is made warp-uniform so that the warp never splits
+    auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+    };
+    auto issue_s = [&](int ks) {
+      if (leader) {
+        const uint64_t kd = kd0 + (uint64_t)(ks * (kKvBytes >> 4));
+        umma_bf16(tm_s, qd, kd, idesc_s, 0u);
+        umma_bf16(tm_s, qd + 2, kd + 2, idesc_s, 1u);
+        umma_bf16(tm_s, qd + 4, kd + 4, idesc_s, 1u);
+        umma_bf16(tm_s, qd + 6, kd + 6, idesc_s, 1u);
+        umma_commit(s_full(t));
+      }
+      __syncwarp();
+    };
+    for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
+      const Item w = load_item(meta, ml, it, n_head);
+      if (t == 1 && !w.two) {
+        // nothing to compute for this tile: release the stages in step with the other tile
+        for (int j = 0; ok && j < w.n_kv; ++j) {
+          int ks = kc % kKvStages;
+          if (!wait_all(k_full(ks), (kc / kKvStages) & 1u)) { ok = false; break; }
+          if (leader) mbar_arrive(k_free(ks));
+          ++kc;
+          int vs = vc % kKvStages;
+          if (!wait_all(v_full(vs), (vc / kKvStages) & 1u)) { ok = false; break; }
+          if (leader) mbar_arrive(v_free(vs));
+          ++vc;
+        }
+        if (!ok) break;
+        if (!wait_all(q_full, items & 1u)) { ok = false; break; }
+        if (leader) mbar_arrive(q_free);
+        ++items;
+        continue;
+      }
+      if (!wait_all(q_full, items & 1u)) { ok = false; break; }
+      int ks = kc % kKvStages;
+      if (!wait_all(k_full(ks), (kc / kKvStages) & 1u)) { ok = false; break; }
+      tc_fence_after();
+      issue_s(ks);  // the score buffer is free: its last reader arrived on s_free (waited below)
+      if (leader) umma_commit(k_free(ks));
+      ++kc;
+      for (int j = 0; j < w.n_kv; ++j) {
+        if (!wait_all(s_free(t), g & 1u)) { ok = false; break; }
+        if (j + 1 < w.n_kv) {
+          ks = kc % kKvStages;
+          if (!wait_all(k_full(ks), (kc / kKvStages) & 1u)) { ok = false; break; }
+          tc_fence_after();
+          issue_s(ks);
+          if (leader) umma_commit(k_free(ks));
+          ++kc;
+        }
+        const int vs = vc % kKvStages;
+        if (!wait_all(v_full(vs), (vc / kKvStages) & 1u)) { ok = false; break; }
+        const int k_steps = (min(kTK, w.n - j * kTK) + 15) >> 4;
+        const uint32_t b = g & 1u;
+        if (!wait_all(p_full(t, b), (g >> 1) & 1u)) { ok = false; break; }
+        tc_fence_after();
+        if (leader) {
+          const uint64_t vd = vd0 + (uint64_t)(vs * (kKvBytes >> 4));
+          const uint32_t tm_o = tm_s + 128 + 64 * b, tm_p = tm_s + 64 + 32 * b;
+          // 16 keys per instruction: 8 packed columns of P, 2048 B of V
+          umma_bf16_ts(tm_o, tm_p, vd, idesc_o, 0u);
+          if (k_steps > 1) umma_bf16_ts(tm_o, tm_p + 8, vd + 128, idesc_o, 1u);
+          if (k_steps > 2) umma_bf16_ts(tm_o, tm_p + 16, vd + 256, idesc_o, 1u);
+          if (k_steps > 3) umma_bf16_ts(tm_o, tm_p + 24, vd + 384, idesc_o, 1u);
+          umma_commit(o_full(t, b));
+          umma_commit(v_free(vs));
+        }
+        __syncwarp();
+        ++vc;
+        ++g;
+      }
+      if (!ok) break;
+      if (leader) umma_commit(q_free);
+      ++items;
+    }
+    if (!ok && leader) atomicExch(err_flag, 12);
+  } else if (warp < 8) {
+    // ------------------------------------------------------------------ softmax, one row per thread
+    const int t = warp >> 2;
+    const int r = (warp & 3) * 32 + lane;
+    const uint32_t lane_field = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t ta_s = tmem_base + lane_field + t * 256;
+    const float scale = 0.125f * 1.4426950408889634f;  // 1/sqrt(64), base-2 exponent
+    uint32_t g = 0;  // steps done by this tile (same counter as the MMA issuer's)
+    bool ok = true;
+
+    for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
+      const Item w = load_item(meta, ml, it, n_head);
+      if (t == 1 && !w.two) continue;
+      // a warp whose 32 rows all lie beyond the sequence keeps pace with the barriers only
+      const bool active = w.q0 + t * kTQ + (warp & 3) * 32 < w.n;
+      float o[kHeadDim];
+#pragma unroll
+      for (int i = 0; i < kHeadDim; ++i) o[i] = 0.f;
+      float m_run = -INFINITY, l_run = 0.f;
+
+      // o += (P V of step gp): read the finished product from tensor memory
+      auto fold_output = [&](uint32_t gp, float scale_o) -> bool {
+        bool good = mbar_wait(o_full(t, gp & 1u), (gp >> 1) & 1u, abort_flag);
+        good = __all_sync(0xffffffffu, good);
+        if (!good) return false;
+        tc_fence_after();
+        if (active) {
+          const uint32_t ta_o = ta_s + 128 + 64 * (gp & 1u);
+          uint32_t a[64];  // the score registers are dead by now: all four loads fly together
+          tmem_ld_32x32(ta_o, *reinterpret_cast<uint32_t(*)[32]>(&a[0]));
+          tmem_ld_32x32(ta_o + 32, *reinterpret_cast<uint32_t(*)[32]>(&a[32]));
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 64; ++i) o[i] = (o[i] + __uint_as_float(a[i])) * scale_o;
+        }
+        return true;
+      };
+
+      for (int j = 0; j < w.n_kv; ++j) {
+        ok = mbar_wait(s_full(t), g & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const int kv_valid = min(kTK, w.n - j * kTK);
+        uint32_t sv[64];
+        if (active) {
+          tmem_ld_32x32(ta_s, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+          tmem_ld_32x32(ta_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+          tmem_ld_wait();
+        }
+        tc_fence_before();
+        mbar_arrive(s_free(t));  // the scores are in registers: the next S may overwrite them
+        if (active) {
+          float mx = -INFINITY;
+          if (kv_valid == kTK) {
+#pragma unroll
+            for (int i = 0; i < 64; i += 2)
+              mx = fmaxf(mx, fmaxf(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 64; ++i)
+              if (i < kv_valid) mx = fmaxf(mx, __uint_as_float(sv[i]));
+          }
+          const float m_new = fmaxf(m_run, mx * scale);  // finite: the first key of a step is always valid
+          const float corr = ex2_approx(m_run - m_new);
+          m_run = m_new;
+          float rs = 0.f;
+          const uint32_t ta_p = ta_s + 64 + 32 * (g & 1u);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              float p0 = ex2_approx(fmaf(__uint_as_float(sv[32 * h + 2 * i]), scale, -m_new));
+              float p1 = ex2_approx(fmaf(__uint_as_float(sv[32 * h + 2 * i + 1]), scale, -m_new));
+              if (kv_valid != kTK) {
+                if (32 * h + 2 * i >= kv_valid) p0 = 0.f;
+                if (32 * h + 2 * i + 1 >= kv_valid) p1 = 0.f;
+              }
+              rs += p0 + p1;
+              __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+              pk[i] = *reinterpret_cast<uint32_t*>(&v);
+            }
+            tmem_st_32x16(ta_p + 16 * h, pk);
+          }
+          tmem_st_wait();
+          l_run = l_run * corr + rs;
+          tc_fence_before();
+          mbar_arrive(p_full(t, g & 1u));
+          // fold in the previous step's product (computed against the previous maximum), then
+          // rescale everything to the new maximum
+          if (j > 0) {
+            if (!fold_output(g - 1, corr)) { ok = false; break; }
+          }
+        } else {
+          tc_fence_before();
+          mbar_arrive(p_full(t, g & 1u));
+          if (j > 0) {
+            if (!fold_output(g - 1, 1.0f)) { ok = false; break; }
+          }
+        }
+        ++g;
+      }
+      if (!ok) break;
+      if (!fold_output(g - 1, 1.0f)) { ok = false; break; }
+      const int q = w.q0 + t * kTQ + r;
+      if (q < w.n) {
+        const float inv = 1.0f / l_run;
+        __nv_bfloat16* dst = out + (long)(w.tok0 + q) * d_model + w.head * kHeadDim;
+#pragma unroll
+        for (int gi = 0; gi < 8; ++gi) {
+          __nv_bfloat162 p0 = __floats2bfloat162_rn(o[8 * gi + 0] * inv, o[8 * gi + 1] * inv);
+          __nv_bfloat162 p1 = __floats2bfloat162_rn(o[8 * gi + 2] * inv, o[8 * gi + 3] * inv);
+          __nv_bfloat162 p2 = __floats2bfloat162_rn(o[8 * gi + 4] * inv, o[8 * gi + 5] * inv);
+          __nv_bfloat162 p3 = __floats2bfloat162_rn(o[8 * gi + 6] * inv, o[8 * gi + 7] * inv);
+          uint4 u;
+          u.x = *reinterpret_cast<uint32_t*>(&p0);
+          u.y = *reinterpret_cast<uint32_t*>(&p1);
+          u.z = *reinterpret_cast<uint32_t*>(&p2);
+          u.w = *reinterpret_cast<uint32_t*>(&p3);
+          *reinterpret_cast<uint4*>(dst + 8 * gi) = u;
+        }
+      }
+    }
+    if (!ok && lane == 0) atomicExch(err_flag, 13);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+cudaError_t attention_bf16_configure() {
+  return cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttnSmem);
+}
+
+void launch_attention_bf16(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, __nv_bfloat16* out,
+                           const int* meta, MetaLayout ml, int n_work, int d_model, int* err_flag, int num_sms,
+                           cudaStream_t s) {
+  if (n_work <= 0) return;
+  const int n_head = d_model / kHeadDim;
+  const int n_items = n_work * n_head;
+  const int grid = n_items < num_sms ? n_items : num_sms;
+  attention_tc_kernel<<<grid, kAttnThreads, kAttnSmem, s>>>(tmap_q, tmap_kv, out, meta, ml, n_items, n_head, d_model,
+                                                            err_flag);
+}
+
+}  // namespace wf

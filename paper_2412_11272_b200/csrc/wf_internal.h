@@ -99,9 +99,12 @@ cudaError_t gemm_bf16_configure();
 void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
                       int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s);
 
-// ---- bf16 attention (wf_attention.cu)
+// ---- bf16 attention on tcgen05 (wf_attention_tc.cu); work items are 256 query rows
 cudaError_t attention_bf16_configure();
-void launch_attention_bf16(const __nv_bfloat16* qkv, __nv_bfloat16* out, const int* meta,
-                           MetaLayout ml, int n_work, int d_model, cudaStream_t s);
+// tmap_q / tmap_kv: bf16 [rows, 3 d_model] maps of the same buffer with 64 x 128 and 64 x 64 boxes
+// (make_tmap_bf16 with box_rows 128 and 64)
+void launch_attention_bf16(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, __nv_bfloat16* out,
+                           const int* meta, MetaLayout ml, int n_work, int d_model, int* err_flag, int num_sms,
+                           cudaStream_t s);
 
 }  // namespace wf
