@@ -1,0 +1,101 @@
+"""Runs one component of the library alone, for timing and for profiler captures.
+
+    python -m paper_2412_11272_b200.probe gemm --M 16384 --N 3840 --K 1280 --mode 0
+    python -m paper_2412_11272_b200.probe attention --n 775 --batch 64
+    python -m paper_2412_11272_b200.probe encode --shape large --seconds 3 --batch 16
+    python -m paper_2412_11272_b200.probe logmel --seconds 15 --batch 64
+
+Each command warms up, times ``--iters`` launches with CUDA events on the launching stream and
+prints one JSON line (milliseconds per launch and the algorithmic rate).  Inputs are synthetic.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+
+import numpy as np
+import torch
+
+from . import inputs as I
+from .binding import Encoder
+
+
+def _time(fn, iters, warmup=3):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def _component_encoder(d_model=128, n_head=2, max_batch=1, max_tokens=64):
+    shape = I.EncoderShape("probe", 80, d_model, 0, n_head, 256, "bf16", n_ctx=4096)
+    return Encoder(shape, I.encoder_weights(0, shape), I.mel_filterbank(80), max_batch, max_tokens, 1000)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("what", choices=["gemm", "attention", "encode", "logmel"])
+    ap.add_argument("--M", type=int, default=16384)
+    ap.add_argument("--N", type=int, default=3840)
+    ap.add_argument("--K", type=int, default=1280)
+    ap.add_argument("--mode", type=int, default=0)
+    ap.add_argument("--n", type=int, default=775)
+    ap.add_argument("--batch", type=int, default=64)
+    ap.add_argument("--d_model", type=int, default=1280)
+    ap.add_argument("--shape", default="large")
+    ap.add_argument("--seconds", type=float, default=3.0)
+    ap.add_argument("--iters", type=int, default=10)
+    a = ap.parse_args()
+    out = {"what": a.what}
+    if a.what == "gemm":
+        enc = _component_encoder()
+        A = torch.randn(a.M, a.K, device="cuda").to(torch.bfloat16)
+        W = (torch.randn(a.N, a.K, device="cuda") / math.sqrt(a.K)).to(torch.bfloat16)
+        b = torch.randn(a.N, device="cuda")
+        C = torch.zeros(a.M, a.N, device="cuda", dtype=torch.float32 if a.mode == 2 else torch.bfloat16)
+        ms = _time(lambda: enc.wf_gemm_bf16(A, W, b, a.mode, C), a.iters)
+        enc.wf_check()
+        out.update(M=a.M, N=a.N, K=a.K, mode=a.mode, ms=ms, tflops=2.0 * a.M * a.N * a.K / ms / 1e9)
+    elif a.what == "attention":
+        d = a.d_model
+        enc = _component_encoder(d, d // 64, a.batch, a.batch * a.n)
+        cu = np.arange(a.batch + 1) * a.n
+        qkv = torch.randn(int(cu[-1]), 3 * d, device="cuda").to(torch.bfloat16)
+        ms = _time(lambda: enc.wf_attention(qkv, cu), a.iters)
+        enc.wf_check()
+        out.update(n=a.n, batch=a.batch, d_model=d, ms=ms, tflops=4.0 * a.batch * a.n * a.n * d / ms / 1e9)
+    else:
+        shape = I.SHAPES[a.shape]
+        n_layer = shape.n_layer if a.what == "encode" else 0
+        shape = I.EncoderShape(shape.name, shape.n_mel, shape.d_model, n_layer, shape.n_head, shape.d_mlp,
+                               shape.dtype, shape.n_ctx)
+        L = int(a.seconds * 100) * 160
+        lengths = np.full(a.batch, L, dtype=np.int64)
+        batch = I.batch_from_lengths(0, lengths)
+        audio = torch.as_tensor(batch.audio).cuda()
+        hush = torch.as_tensor(I.round_to_bf16(I.hush_mel(0, shape.n_mel))).cuda()
+        tokens = int(I.tokens_of(lengths).sum())
+        enc = Encoder(shape, I.encoder_weights(0, shape), I.mel_filterbank(shape.n_mel), a.batch, tokens,
+                      int(lengths.sum()))
+        if a.what == "encode":
+            ms = _time(lambda: enc.wf_encode(audio, lengths, hush), a.iters)
+            fl = I.algorithmic_flops(shape, lengths)
+            out.update(shape=a.shape, tokens=tokens, ms=ms, tflops=fl["encoder"] / ms / 1e9)
+        else:
+            ms = _time(lambda: enc.wf_logmel(audio, lengths), a.iters)
+            frames = int((lengths // 160).sum())
+            out.update(frames=frames, ms=ms, gbs=(4.0 * lengths.sum() + 4.0 * frames * shape.n_mel) / ms / 1e6,
+                       fp32_tflops=frames * (2 * 201 * 399 + 2 * 201 * shape.n_mel) / ms / 1e9)
+        enc.wf_check()
+    print(json.dumps(out), flush=True)
+
+
+if __name__ == "__main__":
+    main()
