@@ -506,14 +506,15 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     ok &= make_tmap_out(e->tma, &e->tmo_qkv, e->qkv, 2, 3 * d, mt);
     ok &= make_tmap_out(e->tma, &e->tmo_fc1, e->fc1, 2, F, mt);
     ok &= make_tmap_out(e->tma, &e->tmo_x, e->x, 4, d, mt);
-    ok &= make_tmap_bf16(e->tma, &e->tm_conv1_w, e->conv1_w, 3 * e->mel_ld, d, 3 * e->mel_ld, 256);
-    ok &= make_tmap_bf16(e->tma, &e->tm_conv2_w, e->conv2_w, 3 * d, d, 3 * d, 256);
+    const uint32_t wbox = gemm_bf16_uses_pair() ? 128 : 256;
+    ok &= make_tmap_bf16(e->tma, &e->tm_conv1_w, e->conv1_w, 3 * e->mel_ld, d, 3 * e->mel_ld, wbox);
+    ok &= make_tmap_bf16(e->tma, &e->tm_conv2_w, e->conv2_w, 3 * d, d, 3 * d, wbox);
     for (int l = 0; l < c.n_layer; ++l) {
       LayerW& L = e->layers[l];
-      ok &= make_tmap_bf16(e->tma, &L.tm_wqkv, L.wqkv, d, 3 * d, d, 256);
-      ok &= make_tmap_bf16(e->tma, &L.tm_wo, L.wo, d, d, d, 256);
-      ok &= make_tmap_bf16(e->tma, &L.tm_w1, L.w1, d, F, d, 256);
-      ok &= make_tmap_bf16(e->tma, &L.tm_w2, L.w2, F, d, F, 256);
+      ok &= make_tmap_bf16(e->tma, &L.tm_wqkv, L.wqkv, d, 3 * d, d, wbox);
+      ok &= make_tmap_bf16(e->tma, &L.tm_wo, L.wo, d, d, d, wbox);
+      ok &= make_tmap_bf16(e->tma, &L.tm_w1, L.w1, d, F, d, wbox);
+      ok &= make_tmap_bf16(e->tma, &L.tm_w2, L.w2, F, d, F, wbox);
     }
     if (!ok) return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
   }
@@ -655,7 +656,7 @@ wf_status wf_gemm_bf16(wf_encoder* e, const void* A, const void* W, const float*
     return fail(e, WF_ERR_INVALID_ARG, "wf_gemm_bf16: bad pointer, size or mode");
   if (M == 0) return WF_OK;
   CUtensorMap ta, tb, tc;
-  if (!make_tmap_bf16(e->tma, &ta, A, K, M, K, 128) || !make_tmap_bf16(e->tma, &tb, W, K, N, K, 256) ||
+  if (!make_tmap_bf16(e->tma, &ta, A, K, M, K, 128) || !make_tmap_bf16(e->tma, &tb, W, K, N, K, gemm_bf16_uses_pair() ? 128 : 256) ||
       !make_tmap_out(e->tma, &tc, C, mode == 2 ? 4 : 2, N, M))
     return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
   EpiParams ep{};

@@ -74,6 +74,90 @@ __device__ __forceinline__ void conv2_store32(const EpiParams& ep, long row, lon
   }
 }
 
+// Epilogue of one 128 x BN accumulator tile for the warp that owns TMEM lanes 32 * quarter ..:
+// t_row is the tensor-memory address of that lane group's first column of the tile, m0 / n0 the
+// tile origin in the output, stage_base this warp's two 4 KB staging buffers.
+template <int BN, int EPI>
+__device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtensorMap* tmap_c, uint32_t t_row, int m0,
+                                              int n0, long M, int N, int quarter, int lane, uint32_t stage_base,
+                                              uint32_t& piece) {
+  const long row = (long)m0 + quarter * 32 + lane;
+  if (EPI == kEpiConv2) {
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+      uint32_t a32[32];
+      float v[32];
+      tmem_ld_32x32(t_row + c * 32, a32);
+      tmem_ld_wait();
+      bias_act32<EPI>(ep, n0 + c * 32, N, a32, v);
+      conv2_store32(ep, row, M, n0 + c * 32, N, v);
+    }
+  } else if (EPI == kEpiBiasResid) {
+    // float32: 32 columns = 128 bytes per row and piece
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+      const uint32_t buf = stage_base + (uint32_t)((piece & 1) * 4096);
+      if (lane == 0) bulk_wait_read<1>();   // the copy that last read this buffer is done with it
+      __syncwarp();
+      uint32_t a32[32];
+      float v[32];
+      tmem_ld_32x32(t_row + c * 32, a32);
+      tmem_ld_wait();
+      bias_act32<EPI>(ep, n0 + c * 32, N, a32, v);
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        st_shared_v4(buf + lane * 128 + ((j ^ (lane & 7)) << 4), __float_as_uint(v[4 * j]),
+                     __float_as_uint(v[4 * j + 1]), __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0 && n0 + c * 32 < N && (long)m0 + quarter * 32 < M) {
+        tma_reduce_add_2d(tmap_c, buf, n0 + c * 32, m0 + quarter * 32);
+        bulk_commit();
+      }
+      ++piece;
+    }
+  } else {
+    // bf16: 64 columns = 128 bytes per row and piece
+    bool valid = true;
+    if (EPI == kEpiConv1) valid = row < M && ep.row_valid[row] != 0;
+#pragma unroll 1
+    for (int c = 0; c < BN / 64; ++c) {
+      const uint32_t buf = stage_base + (uint32_t)((piece & 1) * 4096);
+      if (lane == 0) bulk_wait_read<1>();
+      __syncwarp();
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t a32[32];
+        float v[32];
+        tmem_ld_32x32(t_row + c * 64 + hf * 32, a32);
+        tmem_ld_wait();
+        bias_act32<EPI>(ep, n0 + c * 64 + hf * 32, N, a32, v);
+        if (EPI == kEpiConv1 && !valid) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          __nv_bfloat162 p0 = __floats2bfloat162_rn(v[8 * j + 0], v[8 * j + 1]);
+          __nv_bfloat162 p1 = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
+          __nv_bfloat162 p2 = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
+          __nv_bfloat162 p3 = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
+          st_shared_v4(buf + lane * 128 + (((hf * 4 + j) ^ (lane & 7)) << 4), *reinterpret_cast<uint32_t*>(&p0),
+                       *reinterpret_cast<uint32_t*>(&p1), *reinterpret_cast<uint32_t*>(&p2),
+                       *reinterpret_cast<uint32_t*>(&p3));
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0 && n0 + c * 64 < N && (long)m0 + quarter * 32 < M) {
+        tma_store_2d(tmap_c, buf, n0 + c * 64, m0 + quarter * 32);
+        bulk_commit();
+      }
+      ++piece;
+    }
+  }
+}
+
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
     const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -201,82 +285,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
         break;
       }
       tc_fence_after();
-      const long row = (long)m0 + quarter * 32 + lane;
-      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
-      if (EPI == kEpiConv2) {
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t a32[32];
-          float v[32];
-          tmem_ld_32x32(t_row + c * 32, a32);
-          tmem_ld_wait();
-          bias_act32<EPI>(ep, n0 + c * 32, N, a32, v);
-          conv2_store32(ep, row, M, n0 + c * 32, N, v);
-        }
-      } else if (EPI == kEpiBiasResid) {
-        // float32: 32 columns = 128 bytes per row and piece
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          const uint32_t buf = stage_base + (uint32_t)((piece & 1) * 4096);
-          if (lane == 0) bulk_wait_read<1>();   // the copy that last read this buffer is done with it
-          __syncwarp();
-          uint32_t a32[32];
-          float v[32];
-          tmem_ld_32x32(t_row + c * 32, a32);
-          tmem_ld_wait();
-          bias_act32<EPI>(ep, n0 + c * 32, N, a32, v);
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            st_shared_v4(buf + lane * 128 + ((j ^ (lane & 7)) << 4), __float_as_uint(v[4 * j]),
-                         __float_as_uint(v[4 * j + 1]), __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0 && n0 + c * 32 < N && (long)m0 + quarter * 32 < M) {
-            tma_reduce_add_2d(&tmap_c, buf, n0 + c * 32, m0 + quarter * 32);
-            bulk_commit();
-          }
-          ++piece;
-        }
-      } else {
-        // bf16: 64 columns = 128 bytes per row and piece
-        bool valid = true;
-        if (EPI == kEpiConv1) valid = row < M && ep.row_valid[row] != 0;
-#pragma unroll 1
-        for (int c = 0; c < BN / 64; ++c) {
-          const uint32_t buf = stage_base + (uint32_t)((piece & 1) * 4096);
-          if (lane == 0) bulk_wait_read<1>();
-          __syncwarp();
-#pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            uint32_t a32[32];
-            float v[32];
-            tmem_ld_32x32(t_row + c * 64 + hf * 32, a32);
-            tmem_ld_wait();
-            bias_act32<EPI>(ep, n0 + c * 64 + hf * 32, N, a32, v);
-            if (EPI == kEpiConv1 && !valid) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) v[i] = 0.f;
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              __nv_bfloat162 p0 = __floats2bfloat162_rn(v[8 * j + 0], v[8 * j + 1]);
-              __nv_bfloat162 p1 = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
-              __nv_bfloat162 p2 = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
-              __nv_bfloat162 p3 = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
-              st_shared_v4(buf + lane * 128 + (((hf * 4 + j) ^ (lane & 7)) << 4), *reinterpret_cast<uint32_t*>(&p0),
-                           *reinterpret_cast<uint32_t*>(&p1), *reinterpret_cast<uint32_t*>(&p2),
-                           *reinterpret_cast<uint32_t*>(&p3));
-            }
-          }
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0 && n0 + c * 64 < N && (long)m0 + quarter * 32 < M) {
-            tma_store_2d(&tmap_c, buf, n0 + c * 64, m0 + quarter * 32);
-            bulk_commit();
-          }
-          ++piece;
-        }
-      }
+      epilogue_tile<BN, EPI>(ep, &tmap_c, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN), m0, n0,
+                             M, N, quarter, lane, stage_base, piece);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
@@ -290,6 +300,153 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same GEMM on CTA pairs (thread-block clusters of two, tcgen05 cta_group::2): one MMA
+// covers a 256 x 256 tile, 128 rows per CTA, and each CTA stages only half of the W tile
+// (128 of the 256 output columns), which cuts the shared-memory traffic per flop by a third.
+//   - both CTAs run a TMA producer for their own halves; every copy signals the full barrier
+//     of the pair's first CTA (the leader), which alone issues the MMAs;
+//   - tcgen05.commit multicasts "stage free" and "accumulator ready" to both CTAs;
+//   - the epilogue warps of both CTAs arrive on the leader's "accumulator drained" barrier.
+template <int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
+    const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+    const __grid_constant__ CUtensorMap tmap_c, long M, int N, int K, int a_cols, EpiParams ep, int* err_flag) {
+  constexpr int BN = 256;
+  constexpr int kStages = 6;
+  constexpr int kABytes = kBM * kBK * 2;          // this CTA's 128 rows of A
+  constexpr int kBBytes = (BN / 2) * kBK * 2;     // this CTA's 128 of the 256 W rows
+  constexpr int kStageBytes = kABytes + kBBytes;  // 32 KB
+  constexpr int kStagingOffset = kStages * kStageBytes;
+  constexpr int kBarOffset = kStagingOffset + 4 * 2 * 4096;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + kBarOffset;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + kBarOffset + 8 * (2 * kStages + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + kBarOffset + 8 * (2 * kStages + 4) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // 0 = leader
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);    // used in the leader only: its producer's arrive + both CTAs' bytes
+      mbar_init(empty_bar(s), 1);   // one multicast commit
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);   // one multicast commit
+      mbar_init(tempty_bar(a), 8);  // used in the leader only: 4 epilogue warps of each CTA
+    }
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  cluster_sync_all();  // barriers of both CTAs are initialised before anyone signals them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int num_m = (int)((M + 2 * kBM - 1) / (2 * kBM));
+  const int num_n = (N + BN - 1) / BN;
+  const int num_k = (K + kBK - 1) / kBK;
+  const int num_tiles = num_m * num_n;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&tmap_a);
+      prefetch_tmap(&tmap_b);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair_id; ok && tile < num_tiles; tile += n_pairs) {
+        const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
+        const int n0 = (tile % num_n) * BN + (int)rank * (BN / 2);
+        for (int kb = 0; kb < num_k; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t leader_full = map_to_cta(full_bar(stage), 0);  // the leader CTA's barrier
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * kStageBytes);
+          const uint32_t sa = smem_base + stage * kStageBytes;
+          const int e = kb * kBK;
+          tma_load_2d_pair(sa, &tmap_a, e % a_cols, m0 + e / a_cols, leader_full);
+          tma_load_2d_pair(sa + kABytes, &tmap_b, kb * kBK, n0, leader_full);
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) atomicExch(err_flag, 4);
+    }
+  } else if (warp == 1) {
+    if (rank == 0 && lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(2 * kBM, BN, 0, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = pair_id; ok && tile < num_tiles; tile += n_pairs) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_k; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * kStageBytes;
+          const uint64_t adesc = umma_desc_k_sw128(sa);
+          const uint64_t bdesc = umma_desc_k_sw128(sa + kABytes);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)
+            umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          umma_commit_pair(empty_bar(stage), 3);
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit_pair(tfull_bar(acc), 3);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (!ok) atomicExch(err_flag, 5);
+    }
+  } else {
+    const int quarter = warp & 3;
+    const uint32_t stage_base = smem_base + kStagingOffset + (uint32_t)((warp - 2) * 8192);
+    uint32_t piece = 0;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = pair_id; tile < num_tiles; tile += n_pairs) {
+      const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
+      const int n0 = (tile % num_n) * BN;
+      bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) {
+        if (lane == 0) atomicExch(err_flag, 6);
+        break;
+      }
+      tc_fence_after();
+      epilogue_tile<BN, EPI>(ep, &tmap_c, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN), m0, n0,
+                             M, N, quarter, lane, stage_base, piece);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+    if (lane == 0) bulk_wait_all();
+  }
+
+  tc_fence_before();
+  cluster_sync_all();  // neither CTA leaves while the other may still touch its memory or barriers
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 512);
   }
 }
 
@@ -337,8 +494,23 @@ static cudaError_t configure_one() {
                               GemmCfg<BN>::kSmemBytes);
 }
 
+constexpr int kPairSmemBytes = 6 * 32768 + 4 * 2 * 4096 + 256 + 1024;
+
+template <int EPI>
+static cudaError_t configure_pair() {
+  cudaError_t e = cudaFuncSetAttribute(gemm_bf16_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kPairSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_bf16_pair_kernel<EPI>, cudaFuncAttributeNonPortableClusterSizeAllowed, 0);
+}
+
 cudaError_t gemm_bf16_configure() {
   cudaError_t e;
+  if ((e = configure_pair<kEpiBias>()) != cudaSuccess) return e;
+  if ((e = configure_pair<kEpiBiasGelu>()) != cudaSuccess) return e;
+  if ((e = configure_pair<kEpiBiasResid>()) != cudaSuccess) return e;
+  if ((e = configure_pair<kEpiConv1>()) != cudaSuccess) return e;
+  if ((e = configure_pair<kEpiConv2>()) != cudaSuccess) return e;
   if ((e = configure_one<256, kEpiBias>()) != cudaSuccess) return e;
   if ((e = configure_one<256, kEpiBiasGelu>()) != cudaSuccess) return e;
   if ((e = configure_one<256, kEpiBiasResid>()) != cudaSuccess) return e;
@@ -356,9 +528,44 @@ static void launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUten
                                                                                  err_flag);
 }
 
+template <int EPI>
+static void launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
+                        int a_cols, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
+  const long tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + 255) / 256);
+  const long pairs = tiles < num_sms / 2 ? tiles : num_sms / 2;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = kPairSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, gemm_bf16_pair_kernel<EPI>, ta, tb, tc, M, N, K, a_cols, ep, err_flag);
+}
+
+// pair = 1: CTA-pair kernel (W maps must then use 128-row boxes); 0: single-CTA kernel
+static int g_gemm_use_pair = 1;
+void gemm_bf16_set_pair(int on) { g_gemm_use_pair = on; }
+int gemm_bf16_uses_pair() { return g_gemm_use_pair; }
+
 void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
                       int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
   if (M <= 0 || N <= 0 || K <= 0) return;
+  if (g_gemm_use_pair) {
+    switch (epi) {
+      case kEpiBias: launch_pair<kEpiBias>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+      case kEpiBiasGelu: launch_pair<kEpiBiasGelu>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+      case kEpiBiasResid: launch_pair<kEpiBiasResid>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+      case kEpiConv1: launch_pair<kEpiConv1>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+      default: launch_pair<kEpiConv2>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    }
+    return;
+  }
   switch (epi) {
     case kEpiBias: launch_one<256, kEpiBias>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
     case kEpiBiasGelu: launch_one<256, kEpiBiasGelu>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;

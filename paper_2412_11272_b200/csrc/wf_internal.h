@@ -91,6 +91,9 @@ bool make_tmap_bf16(const TmaApi& api, CUtensorMap* m, const void* base, uint64_
 bool make_tmap_out(const TmaApi& api, CUtensorMap* m, const void* base, int elem_bytes, uint64_t cols,
                    uint64_t rows);
 cudaError_t gemm_bf16_configure();
+// 1 (default): CTA-pair kernel, W tensor maps need 128-row boxes; 0: single-CTA kernel, 256-row boxes
+int gemm_bf16_uses_pair();
+void gemm_bf16_set_pair(int on);
 // a_cols: stored row length of A in elements (K for a plain GEMM; smaller when one GEMM row
 // spans several consecutive stored rows, which must then be a multiple of 64).
 // tc: output map (bf16 out for kEpiBias/kEpiBiasGelu/kEpiConv1, float32 residual for
