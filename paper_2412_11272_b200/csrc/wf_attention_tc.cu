@@ -309,8 +309,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
         }
         tc_fence_before();
         mbar_arrive(s_free(t));  // the scores are in registers: the next S may overwrite them
+        float mx = -INFINITY, corr = 1.0f, m_new = m_run;
         if (active) {
-          float mx = -INFINITY;
           if (kv_valid == kTK) {
 #pragma unroll
             for (int i = 0; i < 64; i += 2)
@@ -320,9 +320,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
             for (int i = 0; i < 64; ++i)
               if (i < kv_valid) mx = fmaxf(mx, __uint_as_float(sv[i]));
           }
-          const float m_new = fmaxf(m_run, mx * scale);  // finite: the first key of a step is always valid
-          const float corr = ex2_approx(m_run - m_new);
+          m_new = fmaxf(m_run, mx * scale);  // finite: the first key of a step is always valid
+          corr = ex2_approx(m_run - m_new);
           m_run = m_new;
+        }
+        if (active) {
           float rs = 0.f;
           const uint32_t ta_p = ta_s + 64 + 32 * (g & 1u);
 #pragma unroll
@@ -342,21 +344,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
             }
             tmem_st_32x16(ta_p + 16 * h, pk);
           }
-          tmem_st_wait();
           l_run = l_run * corr + rs;
-          tc_fence_before();
-          mbar_arrive(p_full(t, g & 1u));
-          // fold in the previous step's product (computed against the previous maximum), then
-          // rescale everything to the new maximum
-          if (j > 0) {
-            if (!fold_output(g - 1, corr)) { ok = false; break; }
-          }
-        } else {
-          tc_fence_before();
-          mbar_arrive(p_full(t, g & 1u));
-          if (j > 0) {
-            if (!fold_output(g - 1, 1.0f)) { ok = false; break; }
-          }
+        }
+        if (active) tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(p_full(t, g & 1u));
+        // fold in the previous step's product (computed against the previous maximum) and rescale
+        // everything to the new maximum
+        if (j > 0) {
+          if (!fold_output(g - 1, corr)) { ok = false; break; }
         }
         ++g;
       }
