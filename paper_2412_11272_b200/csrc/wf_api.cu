@@ -45,7 +45,7 @@ struct wf_encoder {
   std::vector<LayerW> layers;
   CUtensorMap tm_conv1_w, tm_conv2_w, tm_zp, tm_c1p, tm_h, tm_attn, tm_fc1;
   CUtensorMap tmo_c1p, tmo_qkv, tmo_fc1, tmo_x;  // epilogue outputs
-  CUtensorMap tm_qkv, tm_qkv_kv;                 // attention operand loads (128- and 64-row boxes)
+  CUtensorMap tm_qkv, tm_qkv_kv;                 // attention operand loads (128- and 96-row boxes)
 
   float* logmel;
   int* seq_max;
@@ -501,7 +501,7 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     ok &= make_tmap_bf16(e->tma, &e->tm_attn, e->attn, d, mt, d, 128);
     ok &= make_tmap_bf16(e->tma, &e->tm_fc1, e->fc1, F, mt, F, 128);
     ok &= make_tmap_bf16(e->tma, &e->tm_qkv, e->qkv, 3 * d, mt, 3 * d, 128);
-    ok &= make_tmap_bf16(e->tma, &e->tm_qkv_kv, e->qkv, 3 * d, mt, 3 * d, 64);
+    ok &= make_tmap_bf16(e->tma, &e->tm_qkv_kv, e->qkv, 3 * d, mt, 3 * d, 96);
     ok &= make_tmap_out(e->tma, &e->tmo_c1p, e->c1p, 2, d, e->cap_prows + 4);
     ok &= make_tmap_out(e->tma, &e->tmo_qkv, e->qkv, 2, 3 * d, mt);
     ok &= make_tmap_out(e->tma, &e->tmo_fc1, e->fc1, 2, F, mt);
@@ -704,7 +704,7 @@ wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, in
     if (e->bf16) {
       CUtensorMap tq, tkv;
       if (!make_tmap_bf16(e->tma, &tq, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 128) ||
-          !make_tmap_bf16(e->tma, &tkv, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 64))
+          !make_tmap_bf16(e->tma, &tkv, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 96))
         return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected the qkv tensor map");
       launch_attention_bf16(tq, tkv, (__nv_bfloat16*)out, e->meta_dev[slot], ml, nw, e->cfg.d_model, e->err_flag, e->num_sms, s);
     }

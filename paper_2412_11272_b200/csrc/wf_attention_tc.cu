@@ -1,26 +1,29 @@
 // Non-causal variable-length attention on the 5th-generation tensor cores (bf16, head dim 64).
 //
 // A persistent CTA (352 threads) walks a list of work items; one item = up to 256 query rows
-// (two tiles of 128) of one (sequence, head); keys are consumed 64 at a time.  Roles:
+// (two tiles of 128) of one (sequence, head); keys are consumed 96 at a time.  Roles:
 //   warps 0-3 / 4-7  softmax for query tile 0 / 1, one thread per query row.  A step loads the
-//                    64 scores of its row from tensor memory once, releases the score buffer,
-//                    takes the row maximum, exponentiates, writes the probabilities back to
-//                    tensor memory as packed bf16 (double-buffered) and only then folds in the
-//                    P V product of the PREVIOUS step, so it never waits on the tensor pipe in
-//                    steady state.  The running output row lives in registers.
-//   warp 8           one lane issues the TMA loads: Q tiles once per item, K and V tiles of 64
+//                    96 scores of its row from tensor memory once, releases the score buffer,
+//                    takes the row maximum, exponentiates and writes the probabilities back to
+//                    tensor memory as packed bf16 (double-buffered).  The output row is
+//                    accumulated by the tensor core in tensor memory across steps; probabilities
+//                    are taken relative to a reference maximum that is only raised (and the
+//                    accumulator rescaled, read-modify-write in tensor memory) when the true
+//                    maximum exceeds it by more than 2^8 -- the final O / l does not depend on
+//                    that choice.  In steady state the softmax never waits for the tensor pipe.
+//   warp 8           one lane issues the TMA loads: Q tiles once per item, K and V tiles of 96
 //                    keys through two 4-stage rings.
 //   warps 9, 10      MMA issue for query tile 0 / 1 (warp 9 also owns the tensor-memory
 //                    allocation).  The whole warp runs the loop so that descriptors stay in
-//                    uniform registers; one elected lane issues S = Q K^T (128x64x64, operands in
+//                    uniform registers; one elected lane issues S = Q K^T (128x96x64, operands in
 //                    shared memory) as soon as the softmax has read the previous scores, and
-//                    O = P V (128x64x64, P from tensor memory, V from shared memory as an MN-major
-//                    operand) when the probabilities are in place.  A K / V stage is released
-//                    when both tiles' MMAs on it have completed (barriers count two arrivals).
+//                    O += P V (128x64x96, P from tensor memory, V from shared memory as an
+//                    MN-major operand) when the probabilities are in place.  A K / V stage is
+//                    released when both tiles' MMAs on it have completed (barriers count two).
 // Keys are addressed through the token prefix sums: a key tile that runs past the end of its
 // sequence is masked in the softmax, so no padded token ever contributes.
-// Tensor-memory columns per query tile t (base 256 t): S [0,64) f32; P0 [64,96), P1 [96,128)
-// packed bf16; O0 [128,192), O1 [192,256) f32.  Every mbarrier wait is bounded (wf_ptx.cuh).
+// Tensor-memory columns per query tile t (base 256 t): S [0,96) f32; P0 [96,144), P1 [144,192)
+// packed bf16; O [192,256) f32.  Every mbarrier wait is bounded (wf_ptx.cuh).
 #include "wf_internal.h"
 #include "wf_ptx.cuh"
 
@@ -31,10 +34,10 @@ using namespace ptx;
 namespace {
 
 constexpr int kTQ = 128;          // query rows per tile
-constexpr int kTK = 64;           // keys per step
+constexpr int kTK = 96;           // keys per step
 constexpr int kKvStages = 4;
 constexpr int kQBytes = kTQ * 64 * 2;      // 16 KB
-constexpr int kKvBytes = kTK * 64 * 2;     // 8 KB
+constexpr int kKvBytes = kTK * 64 * 2;     // 12 KB
 constexpr int kAttnThreads = 352;
 
 // shared-memory map (offsets from a 1024-byte aligned base)
@@ -239,12 +242,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
         tc_fence_after();
         if (leader) {
           const uint64_t vd = vd0 + (uint64_t)(vs * (kKvBytes >> 4));
-          const uint32_t tm_o = tm_s + 128 + 64 * b, tm_p = tm_s + 64 + 32 * b;
-          // 16 keys per instruction: 8 packed columns of P, 2048 B of V
-          umma_bf16_ts(tm_o, tm_p, vd, idesc_o, 0u);
+          const uint32_t tm_o = tm_s + 192, tm_p = tm_s + 96 + 48 * b;
+          // 16 keys per instruction: 8 packed columns of P, 2048 B of V; the first instruction of
+          // an item overwrites the accumulator, everything after adds to it
+          umma_bf16_ts(tm_o, tm_p, vd, idesc_o, j > 0 ? 1u : 0u);
           if (k_steps > 1) umma_bf16_ts(tm_o, tm_p + 8, vd + 128, idesc_o, 1u);
           if (k_steps > 2) umma_bf16_ts(tm_o, tm_p + 16, vd + 256, idesc_o, 1u);
           if (k_steps > 3) umma_bf16_ts(tm_o, tm_p + 24, vd + 384, idesc_o, 1u);
+          if (k_steps > 4) umma_bf16_ts(tm_o, tm_p + 32, vd + 512, idesc_o, 1u);
+          if (k_steps > 5) umma_bf16_ts(tm_o, tm_p + 40, vd + 640, idesc_o, 1u);
           umma_commit(o_full(t, b));
           umma_commit(v_free(vs));
         }
@@ -267,73 +273,79 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
     uint32_t g = 0;  // steps done by this tile (same counter as the MMA issuer's)
     bool ok = true;
 
+    const uint32_t ta_o = ta_s + 192;
+    constexpr float kRaise = 8.0f;  // the reference maximum is raised when exceeded by 2^8
+    auto wait_warp = [&](uint32_t bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+    };
+
     for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
       const Item w = load_item(meta, ml, it, n_head);
       if (t == 1 && !w.two) continue;
       // a warp whose 32 rows all lie beyond the sequence keeps pace with the barriers only
       const bool active = w.q0 + t * kTQ + (warp & 3) * 32 < w.n;
-      float o[kHeadDim];
-#pragma unroll
-      for (int i = 0; i < kHeadDim; ++i) o[i] = 0.f;
-      float m_run = -INFINITY, l_run = 0.f;
-
-      // o += (P V of step gp): read the finished product from tensor memory
-      auto fold_output = [&](uint32_t gp, float scale_o) -> bool {
-        bool good = mbar_wait(o_full(t, gp & 1u), (gp >> 1) & 1u, abort_flag);
-        good = __all_sync(0xffffffffu, good);
-        if (!good) return false;
-        tc_fence_after();
-        if (active) {
-          const uint32_t ta_o = ta_s + 128 + 64 * (gp & 1u);
-          uint32_t a[64];  // the score registers are dead by now: all four loads fly together
-          tmem_ld_32x32(ta_o, *reinterpret_cast<uint32_t(*)[32]>(&a[0]));
-          tmem_ld_32x32(ta_o + 32, *reinterpret_cast<uint32_t(*)[32]>(&a[32]));
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 64; ++i) o[i] = (o[i] + __uint_as_float(a[i])) * scale_o;
-        }
-        return true;
-      };
+      float m_ref = -INFINITY, l_run = 0.f;
 
       for (int j = 0; j < w.n_kv; ++j) {
-        ok = mbar_wait(s_full(t), g & 1u, abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        if (!wait_warp(s_full(t), g & 1u)) { ok = false; break; }
         tc_fence_after();
         const int kv_valid = min(kTK, w.n - j * kTK);
-        uint32_t sv[64];
+        uint32_t sv[kTK];
         if (active) {
           tmem_ld_32x32(ta_s, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
           tmem_ld_32x32(ta_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+          tmem_ld_32x32(ta_s + 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[64]));
           tmem_ld_wait();
         }
         tc_fence_before();
         mbar_arrive(s_free(t));  // the scores are in registers: the next S may overwrite them
-        float mx = -INFINITY, corr = 1.0f, m_new = m_run;
         if (active) {
+          float mx = -INFINITY;
           if (kv_valid == kTK) {
 #pragma unroll
-            for (int i = 0; i < 64; i += 2)
+            for (int i = 0; i < kTK; i += 2)
               mx = fmaxf(mx, fmaxf(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])));
           } else {
 #pragma unroll
-            for (int i = 0; i < 64; ++i)
+            for (int i = 0; i < kTK; ++i)
               if (i < kv_valid) mx = fmaxf(mx, __uint_as_float(sv[i]));
           }
-          m_new = fmaxf(m_run, mx * scale);  // finite: the first key of a step is always valid
-          corr = ex2_approx(m_run - m_new);
-          m_run = m_new;
-        }
-        if (active) {
-          float rs = 0.f;
-          const uint32_t ta_p = ta_s + 64 + 32 * (g & 1u);
+          const float m_tile = mx * scale;  // finite: the first key of a step is always valid
+          if (j == 0) {
+            m_ref = m_tile;
+          } else {
+            const bool raise = m_tile > m_ref + kRaise;
+            if (__any_sync(0xffffffffu, raise)) {
+              // rescale this warp's accumulator rows; needs the previous P V to have landed
+              if (!wait_warp(o_full(t, (g - 1) & 1u), ((g - 1) >> 1) & 1u)) { ok = false; break; }
+              tc_fence_after();
+              const float corr = raise ? ex2_approx(m_ref - m_tile) : 1.0f;
+              if (raise) { m_ref = m_tile; l_run *= corr; }
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
+              for (int c = 0; c < 4; ++c) {
+                uint32_t a[16];
+                tmem_ld_32x16(ta_o + 16 * c, a);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) a[i] = __float_as_uint(__uint_as_float(a[i]) * corr);
+                tmem_st_32x16(ta_o + 16 * c, a);
+              }
+              tmem_st_wait();
+            }
+          }
+          // the probability buffer of this step was last read by the P V of two steps ago
+          if (j >= 2) {
+            if (!wait_warp(o_full(t, g & 1u), ((g - 2) >> 1) & 1u)) { ok = false; break; }
+          }
+          float rs = 0.f;
+          const uint32_t ta_p = ta_s + 96 + 48 * (g & 1u);
+#pragma unroll
+          for (int h = 0; h < 3; ++h) {
             uint32_t pk[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              float p0 = ex2_approx(fmaf(__uint_as_float(sv[32 * h + 2 * i]), scale, -m_new));
-              float p1 = ex2_approx(fmaf(__uint_as_float(sv[32 * h + 2 * i + 1]), scale, -m_new));
+              float p0 = ex2_approx(fmaf(__uint_as_float(sv[32 * h + 2 * i]), scale, -m_ref));
+              float p1 = ex2_approx(fmaf(__uint_as_float(sv[32 * h + 2 * i + 1]), scale, -m_ref));
               if (kv_valid != kTK) {
                 if (32 * h + 2 * i >= kv_valid) p0 = 0.f;
                 if (32 * h + 2 * i + 1 >= kv_valid) p1 = 0.f;
@@ -344,38 +356,50 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
             }
             tmem_st_32x16(ta_p + 16 * h, pk);
           }
-          l_run = l_run * corr + rs;
+          l_run += rs;
+          tmem_st_wait();
+        } else if (j >= 2) {
+          if (!wait_warp(o_full(t, g & 1u), ((g - 2) >> 1) & 1u)) { ok = false; break; }
         }
-        if (active) tmem_st_wait();
         tc_fence_before();
         mbar_arrive(p_full(t, g & 1u));
-        // fold in the previous step's product (computed against the previous maximum) and rescale
-        // everything to the new maximum
-        if (j > 0) {
-          if (!fold_output(g - 1, corr)) { ok = false; break; }
-        }
         ++g;
       }
       if (!ok) break;
-      if (!fold_output(g - 1, 1.0f)) { ok = false; break; }
+      // drain the last two products (each barrier phase is waited for exactly in order)
+      if (w.n_kv >= 2) {
+        if (!wait_warp(o_full(t, (g - 2) & 1u), ((g - 2) >> 1) & 1u)) { ok = false; break; }
+      }
+      if (!wait_warp(o_full(t, (g - 1) & 1u), ((g - 1) >> 1) & 1u)) { ok = false; break; }
+      tc_fence_after();
       const int q = w.q0 + t * kTQ + r;
-      if (q < w.n) {
+      if (active) {
         const float inv = 1.0f / l_run;
         __nv_bfloat16* dst = out + (long)(w.tok0 + q) * d_model + w.head * kHeadDim;
 #pragma unroll
-        for (int gi = 0; gi < 8; ++gi) {
-          __nv_bfloat162 p0 = __floats2bfloat162_rn(o[8 * gi + 0] * inv, o[8 * gi + 1] * inv);
-          __nv_bfloat162 p1 = __floats2bfloat162_rn(o[8 * gi + 2] * inv, o[8 * gi + 3] * inv);
-          __nv_bfloat162 p2 = __floats2bfloat162_rn(o[8 * gi + 4] * inv, o[8 * gi + 5] * inv);
-          __nv_bfloat162 p3 = __floats2bfloat162_rn(o[8 * gi + 6] * inv, o[8 * gi + 7] * inv);
-          uint4 u;
-          u.x = *reinterpret_cast<uint32_t*>(&p0);
-          u.y = *reinterpret_cast<uint32_t*>(&p1);
-          u.z = *reinterpret_cast<uint32_t*>(&p2);
-          u.w = *reinterpret_cast<uint32_t*>(&p3);
-          *reinterpret_cast<uint4*>(dst + 8 * gi) = u;
+        for (int c = 0; c < 4; ++c) {
+          uint32_t a[16];
+          tmem_ld_32x16(ta_o + 16 * c, a);
+          tmem_ld_wait();
+          if (q < w.n) {
+#pragma unroll
+            for (int gi = 0; gi < 2; ++gi) {
+              __nv_bfloat162 p0 = __floats2bfloat162_rn(__uint_as_float(a[8 * gi + 0]) * inv, __uint_as_float(a[8 * gi + 1]) * inv);
+              __nv_bfloat162 p1 = __floats2bfloat162_rn(__uint_as_float(a[8 * gi + 2]) * inv, __uint_as_float(a[8 * gi + 3]) * inv);
+              __nv_bfloat162 p2 = __floats2bfloat162_rn(__uint_as_float(a[8 * gi + 4]) * inv, __uint_as_float(a[8 * gi + 5]) * inv);
+              __nv_bfloat162 p3 = __floats2bfloat162_rn(__uint_as_float(a[8 * gi + 6]) * inv, __uint_as_float(a[8 * gi + 7]) * inv);
+              uint4 u;
+              u.x = *reinterpret_cast<uint32_t*>(&p0);
+              u.y = *reinterpret_cast<uint32_t*>(&p1);
+              u.z = *reinterpret_cast<uint32_t*>(&p2);
+              u.w = *reinterpret_cast<uint32_t*>(&p3);
+              *reinterpret_cast<uint4*>(dst + 16 * c + 8 * gi) = u;
+            }
+          }
         }
       }
+      // the accumulator has been read: the next item's first P V may overwrite it
+      tc_fence_before();
     }
     if (!ok && lane == 0) atomicExch(err_flag, 13);
   }

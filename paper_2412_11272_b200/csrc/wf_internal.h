@@ -104,8 +104,8 @@ void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtens
 
 // ---- bf16 attention on tcgen05 (wf_attention_tc.cu); work items are 256 query rows
 cudaError_t attention_bf16_configure();
-// tmap_q / tmap_kv: bf16 [rows, 3 d_model] maps of the same buffer with 64 x 128 and 64 x 64 boxes
-// (make_tmap_bf16 with box_rows 128 and 64)
+// tmap_q / tmap_kv: bf16 [rows, 3 d_model] maps of the same buffer with 64 x 128 and 64 x 96 boxes
+// (make_tmap_bf16 with box_rows 128 and 96)
 void launch_attention_bf16(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, __nv_bfloat16* out,
                            const int* meta, MetaLayout ml, int n_work, int d_model, int* err_flag, int num_sms,
                            cudaStream_t s);
