@@ -144,9 +144,9 @@ def run_reference(args, rank):
 
 def run_ours(args, rank, world, local_rank):
     import torch
-    import torch.distributed as dist
 
     from paper_2412_11272_b200 import build as B
+    from paper_2412_11272_b200 import sharding
     from paper_2412_11272_b200.binding import Encoder
 
     B.build()
@@ -160,7 +160,7 @@ def run_ours(args, rank, world, local_rank):
     hush = torch.as_tensor(hush_np).to(dev)
 
     # this rank's 64 streams (stream ids continue across ranks: weak scaling, no exchange)
-    streams = np.stack([I.large_stream(seed, rank * N_STREAMS + s) for s in range(N_STREAMS)])
+    streams = np.stack([I.large_stream(seed, s) for s in sharding.rank_stream_ids(rank, N_STREAMS)])
     max_tokens = int(I.tokens_of([15 * I.SAMPLE_RATE] * N_STREAMS).sum())
     max_samples = N_STREAMS * 15 * I.SAMPLE_RATE
     enc = Encoder(shape, W, F, N_STREAMS, max_tokens, max_samples, device=dev)
@@ -194,16 +194,11 @@ def run_ours(args, rank, world, local_rank):
             enc.wf_encode_host(audio_host[k], lengths[k], hush, out_host)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        sharding.barrier()
         torch.cuda.synchronize()
 
     def max_over_ranks(x):
-        if world > 1:
-            t = torch.tensor([x], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return x
+        return sharding.max_over_ranks(x, dev)
 
     for _ in range(max(args.warmup, 3)):
         step()

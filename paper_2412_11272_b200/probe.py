@@ -4,6 +4,7 @@
     python -m paper_2412_11272_b200.probe attention --n 775 --batch 64
     python -m paper_2412_11272_b200.probe encode --shape large --seconds 3 --batch 16
     python -m paper_2412_11272_b200.probe logmel --seconds 15 --batch 64
+    python -m paper_2412_11272_b200.probe config --name small        (tiny, base, small, medium-padded, medium-hush, large)
 
 Each command warms up, times ``--iters`` launches with CUDA events on the launching stream and
 prints one JSON line (milliseconds per launch and the algorithmic rate).  Inputs are synthetic.
@@ -41,7 +42,8 @@ def _component_encoder(d_model=128, n_head=2, max_batch=1, max_tokens=64):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["gemm", "attention", "encode", "logmel"])
+    ap.add_argument("what", choices=["gemm", "attention", "encode", "logmel", "config"])
+    ap.add_argument("--name", default="base")
     ap.add_argument("--M", type=int, default=16384)
     ap.add_argument("--N", type=int, default=3840)
     ap.add_argument("--K", type=int, default=1280)
@@ -71,6 +73,40 @@ def main():
         ms = _time(lambda: enc.wf_attention(qkv, cu), a.iters)
         enc.wf_check()
         out.update(n=a.n, batch=a.batch, d_model=d, ms=ms, tflops=4.0 * a.batch * a.n * a.n * d / ms / 1e9)
+    elif a.what == "config":
+        # one named configuration end to end (device-resident inputs), per-call times with CUDA events
+        base = a.name.split("-")[0]
+        shape = I.SHAPES[base]
+        seed = I.CONFIG_SEED[base]
+        kw = {"variant": a.name.split("-")[1]} if base == "medium" else {}
+        hush_frames = 0 if a.name == "medium-padded" else 50
+        batch = I.config_batch(base, **kw)
+        tokens = int(I.tokens_of(batch.lengths, hush_frames).sum())
+        enc = Encoder(shape, I.encoder_weights(seed, shape), I.mel_filterbank(shape.n_mel), len(batch.lengths),
+                      tokens, int(batch.lengths.sum()), hush_frames=hush_frames)
+        audio = torch.as_tensor(batch.audio).cuda()
+        hush = torch.as_tensor(I.round_to_bf16(I.hush_mel(seed, shape.n_mel))).cuda() if hush_frames else None
+        outb = torch.empty((tokens, shape.d_model), dtype=enc.out_dtype, device="cuda")
+        for _ in range(10):
+            enc.wf_encode(audio, batch.lengths, hush, out=outb)
+        torch.cuda.synchronize()
+        evs = []
+        for _ in range(max(a.iters, 50)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            enc.wf_encode(audio, batch.lengths, hush, out=outb)
+            e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        enc.wf_check()
+        times = sorted(x.elapsed_time(y) for x, y in evs)
+        ms = times[len(times) // 2]
+        fl = I.algorithmic_flops(shape, batch.lengths, hush_frames)
+        real_s = batch.meta.get("real_samples", int(batch.lengths.sum())) / I.SAMPLE_RATE
+        out.update(name=a.name, dtype=shape.dtype, batch=len(batch.lengths), tokens=tokens, p50_ms_per_call=ms,
+                   p50_ms_per_buffer=ms / len(batch.lengths), p90_ms_per_call=times[int(len(times) * 0.9)],
+                   audio_s_per_s=real_s / ms * 1e3, tokens_per_s=tokens / ms * 1e3,
+                   tflops=fl["encoder"] / ms / 1e9, gflop_per_call=fl["encoder"] / 1e9)
     else:
         shape = I.SHAPES[a.shape]
         n_layer = shape.n_layer if a.what == "encode" else 0

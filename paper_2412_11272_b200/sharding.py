@@ -1,0 +1,49 @@
+"""Host-side helpers for running the encoder on several GPUs, one process per GPU.
+
+Sequences are independent (no operation of the path crosses a sequence boundary), so the path
+shards without any exchange of activations: weights are replicated, every rank encodes its own
+sequences, and the only collectives are the barrier and the max-reduction of the timing.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+import torch.distributed as dist
+
+
+def rank_stream_ids(rank: int, streams_per_rank: int) -> list[int]:
+    """Weak scaling: rank r owns streams r*S .. r*S + S - 1 (ids are global, never shared)."""
+    return list(range(rank * streams_per_rank, (rank + 1) * streams_per_rank))
+
+
+def sequence_cost(n_tokens, d_model: int, d_mlp: int, n_layer: int) -> np.ndarray:
+    """Algorithmic FLOPs of encoding sequences of n_tokens tokens (GEMMs + attention)."""
+    n = np.asarray(n_tokens, dtype=np.float64)
+    return n_layer * (n * (8.0 * d_model * d_model + 4.0 * d_model * d_mlp) + 4.0 * n * n * d_model)
+
+
+def lpt_partition(costs, world: int) -> list[list[int]]:
+    """Strong scaling of one ragged batch: longest-processing-time-first assignment of sequences
+    to ranks.  Returns, for every rank, the indices of its sequences in their original order."""
+    costs = np.asarray(costs, dtype=np.float64)
+    load = np.zeros(world)
+    parts: list[list[int]] = [[] for _ in range(world)]
+    for i in np.argsort(-costs, kind="stable"):
+        r = int(np.argmin(load))
+        parts[r].append(int(i))
+        load[r] += costs[i]
+    return [sorted(p) for p in parts]
+
+
+def max_over_ranks(value: float, device="cpu") -> float:
+    """The slowest rank's time: what a multi-GPU throughput has to be computed from."""
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier():
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
