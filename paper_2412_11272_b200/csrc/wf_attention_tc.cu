@@ -302,9 +302,16 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
         if (active) {
           float mx = -INFINITY;
           if (kv_valid == kTK) {
+            // four independent chains: a single running maximum would serialise 48 dependent ops
+            float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < kTK; i += 2)
-              mx = fmaxf(mx, fmaxf(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])));
+            for (int i = 0; i < kTK; i += 8) {
+              m0 = fmaxf(m0, fmaxf(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])));
+              m1 = fmaxf(m1, fmaxf(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])));
+              m2 = fmaxf(m2, fmaxf(__uint_as_float(sv[i + 4]), __uint_as_float(sv[i + 5])));
+              m3 = fmaxf(m3, fmaxf(__uint_as_float(sv[i + 6]), __uint_as_float(sv[i + 7])));
+            }
+            mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
           } else {
 #pragma unroll
             for (int i = 0; i < kTK; ++i)
@@ -337,7 +344,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
           if (j >= 2) {
             if (!wait_warp(o_full(t, g & 1u), ((g - 2) >> 1) & 1u)) { ok = false; break; }
           }
-          float rs = 0.f;
+          float rs = 0.f, rs1 = 0.f;
           const uint32_t ta_p = ta_s + 96 + 48 * (g & 1u);
 #pragma unroll
           for (int h = 0; h < 3; ++h) {
@@ -350,13 +357,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
                 if (32 * h + 2 * i >= kv_valid) p0 = 0.f;
                 if (32 * h + 2 * i + 1 >= kv_valid) p1 = 0.f;
               }
-              rs += p0 + p1;
+              if (i & 1) rs1 += p0 + p1; else rs += p0 + p1;
               __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
               pk[i] = *reinterpret_cast<uint32_t*>(&v);
             }
             tmem_st_32x16(ta_p + 16 * h, pk);
           }
-          l_run += rs;
+          l_run += rs + rs1;
           tmem_st_wait();
         } else if (j >= 2) {
           if (!wait_warp(o_full(t, g & 1u), ((g - 2) >> 1) & 1u)) { ok = false; break; }
