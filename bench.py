@@ -33,6 +33,9 @@ UNIT = "audio-s/s"
 WORKLOAD = "large-v3-shaped bf16 encoder, 64 streams x windows of 1..15 s + 50 hush frames (15 ragged calls per step)"
 N_STREAMS = 64
 ROUNDS = list(range(1, 16))
+# DRAM bytes per token of the four block GEMMs (QKV, out-proj, FC1, FC2), from the ncu capture
+# summarised in profiles/gemm_bf16_pair_M16384.md (M = 16384; traffic grows in proportion to M)
+GEMM_DRAM_BYTES_PER_TOKEN = (7713.0, 9480.0, 10612.0, 21024.0)
 SAMPLE_SECONDS = 15         # the CPU oracle is timed on stream 0's full 15 s window (775 tokens)
 
 
@@ -263,12 +266,15 @@ def run_ours(args, rank, world, local_rank):
                 "d2h_bytes_per_step": int(step_tokens * shape.d_model * 2)},
         "gpu_launches": int(launches),
         "kernel_ms_per_step": {k: v["ms"] / args.steps for k, v in prof.items()},
-        "roofline": {"kernel": "gemm_bf16_kernel (tcgen05, QKV / out-proj / FC1 / FC2)", "bound": "tensor",
+        "roofline": {"kernel": "gemm_bf16_pair_kernel (tcgen05 cta_group::2; QKV / out-proj / FC1 / FC2)", "bound": "tensor",
                      "achieved": gemm_tflops, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
                      "frac": (gemm_tflops / peaks["bf16_sustained"]) if gemm_tflops else None,
                      "peak_kind": f"sustained bf16 matmul, {peaks['source']}",
                      "frac_of_burst": (gemm_tflops / peaks["bf16_burst"]) if gemm_tflops else None,
-                     "launches": gemm["launches"], "traffic": None},
+                     "launches": gemm["launches"],
+                     "traffic": sum(GEMM_DRAM_BYTES_PER_TOKEN) / 4.0 * args.steps * step_tokens * shape.n_layer * 4
+                     / max(gemm["launches"], 1),
+                     "traffic_note": "DRAM bytes per launch, scaled per token from the M=16384 ncu capture"},
     }
     if world == 1:
         ref, dt = oracle_sample(W, F, hush_np, seed)
