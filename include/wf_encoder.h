@@ -106,6 +106,18 @@ wf_status wf_logmel(wf_encoder *enc, const float *audio, const long *lengths, in
 wf_status wf_encode(wf_encoder *enc, const float *audio, const long *lengths, int B,
                     const float *hush_mel, void *hidden_out, int *cu_seqlens_out, void *stream);
 
+/* The paper's own variant of the method (Sec. 4.1.2 "Hush word target level", Sec. 5): the hush
+ * word is a raw-audio segment (8000 samples = 0.5 s) that follows the buffer BEFORE the front
+ * end, x (+) h, so frames at the junction straddle both and the per-buffer maximum sees the
+ * hush frames too.  The samples are never copied: the front end reads index i >= L_i of buffer i
+ * from hush_audio[i - L_i].  Needs an encoder created with hush_frames == 0.
+ *   hush_audio    dev  float32 [hush_samples], shared by all buffers; hush_samples <= 16000
+ *   row counts         T_i = floor((L_i + hush_samples) / 160), n_i = ceil(T_i / 2)
+ * Everything else as wf_encode. */
+wf_status wf_encode_raw_hush(wf_encoder *enc, const float *audio, const long *lengths, int B,
+                             const float *hush_audio, int hush_samples, void *hidden_out,
+                             int *cu_seqlens_out, void *stream);
+
 /* Same as wf_encode but starting from normalised log-mel rows (e.g. from wf_logmel, or a
  * raw-audio-level hush word already concatenated by the caller with hush_frames == 0).
  *   mel     dev  float32 [sum T_i, n_mel] packed;   frames  host B row counts T_i >= 1 */

@@ -52,7 +52,7 @@ class wf_weights(C.Structure):
 _PER_LAYER = ("ln1_g", "ln1_b", "wq", "bq", "wk", "wv", "bv", "wo", "bo", "ln2_g", "ln2_b",
               "w1", "b1", "w2", "b2")
 
-EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_mel", "wf_encode_host", "wf_check",
+EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_raw_hush", "wf_encode_mel", "wf_encode_host", "wf_check",
            "wf_encoder_destroy", "wf_last_error", "wf_profile_enable", "wf_profile_read",
            "wf_gemm_bf16", "wf_attention", "wf_attention_f32_static")
 
@@ -72,6 +72,7 @@ def load_library() -> C.CDLL:
     lib.wf_logmel.argtypes = [vp, vp, lp, C.c_int, vp, lp, vp]
     lib.wf_encode.argtypes = [vp, vp, lp, C.c_int, vp, vp, ip, vp]
     lib.wf_encode_mel.argtypes = [vp, vp, lp, C.c_int, vp, vp, ip, vp]
+    lib.wf_encode_raw_hush.argtypes = [vp, vp, lp, C.c_int, vp, C.c_int, vp, ip, vp]
     lib.wf_encode_host.argtypes = [vp, vp, lp, C.c_int, vp, vp, ip, vp]
     lib.wf_check.argtypes = [vp, vp]
     lib.wf_encoder_destroy.argtypes = [vp]
@@ -195,6 +196,20 @@ class Encoder:
                                        hush_mel.data_ptr() if hush_mel is not None else None,
                                        out.data_ptr(), cu.ctypes.data_as(C.POINTER(C.c_int)),
                                        _stream_ptr(stream)))
+        return out, cu
+
+    def wf_encode_raw_hush(self, audio: torch.Tensor, lengths, hush_audio: torch.Tensor, out=None, stream=None):
+        """Hush word at raw-audio level: float32 CUDA samples appended (virtually) to every buffer."""
+        arr, ptr = _longs(lengths)
+        B = len(arr)
+        hs = int(hush_audio.numel())
+        M = int(self._tokens((arr + hs) // 160).sum())
+        if out is None:
+            out = torch.empty((M, self.d_model), dtype=self.out_dtype, device=self.device)
+        cu = np.zeros(B + 1, dtype=np.int32)
+        self._check(self.lib.wf_encode_raw_hush(self.handle, audio.data_ptr() if B else None, ptr, B,
+                                                hush_audio.data_ptr(), hs, out.data_ptr(),
+                                                cu.ctypes.data_as(C.POINTER(C.c_int)), _stream_ptr(stream)))
         return out, cu
 
     def wf_encode_mel(self, mel: torch.Tensor, frames, hush_mel, out=None, stream=None):

@@ -12,6 +12,7 @@ using namespace wf;
 
 namespace {
 constexpr int kRing = 4;          // per-call metadata slots (pinned host + device)
+constexpr int kMaxTailSamples = 16000;  // longest raw-audio hush word (1 s)
 constexpr int kMinSamples = 401;  // reflect padding of 200 needs more than 200 samples on each side
 }  // namespace
 
@@ -34,6 +35,7 @@ struct wf_encoder {
   size_t esz;
   int mel_ld;      // channels per stored log-mel row (n_mel, rounded up to 64 on the bf16 path)
   long cap_prows;  // padded-row capacity
+  long cap_frames; // log-mel rows the front-end scratch holds
   char err[512];
   std::vector<void*> allocs;
   std::vector<void*> pinned;
@@ -159,7 +161,7 @@ class Prof {
 // Builds prefix sums, the padded-row layout and the work lists for one call into `hm`
 // (host ints), validating every length.  `frames_given`: `len` holds frame counts, not samples.
 wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Plan* p, int* hm,
-                    bool build_work = true) {
+                    bool build_work = true, long tail_samples = 0) {
   const wf_config& c = e->cfg;
   if (B < 0 || (B > 0 && !len)) return fail(e, WF_ERR_INVALID_ARG, "bad batch size or NULL lengths");
   if (B > c.max_batch) return fail(e, WF_ERR_CAPACITY, "batch %d exceeds max_batch %d", B, c.max_batch);
@@ -182,7 +184,7 @@ wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Pl
       L = 0;
     } else {
       if (L < kMinSamples) return fail(e, WF_ERR_TOO_SHORT, "buffer %d has %ld samples (need >= %d)", i, L, kMinSamples);
-      T = L / kHop;
+      T = (L + tail_samples) / kHop;  // a raw-audio hush word lengthens every buffer
     }
     long rows = T + c.hush_frames;
     long n = (rows + 1) / 2;
@@ -337,7 +339,8 @@ wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidde
 }
 
 wf_status encode_impl(wf_encoder* e, const float* audio, const float* mel, const long* len, int B,
-                      const float* hush, void* hidden_out, int* cu_out, cudaStream_t s) {
+                      const float* hush, void* hidden_out, int* cu_out, cudaStream_t s,
+                      const float* tail = nullptr, int tail_len = 0) {
   if (!e) return WF_ERR_INVALID_ARG;
   const wf_config& c = e->cfg;
   if (c.hush_frames > 0 && !hush) return fail(e, WF_ERR_INVALID_ARG, "hush_mel is NULL but hush_frames > 0");
@@ -348,7 +351,9 @@ wf_status encode_impl(wf_encoder* e, const float* audio, const float* mel, const
   wf_status st = ring_acquire(e, &slot);
   if (st != WF_OK) return st;
   Plan p;
-  st = make_plan(e, len, mel != nullptr, B, &p, e->meta_host[slot]);
+  st = make_plan(e, len, mel != nullptr, B, &p, e->meta_host[slot], true, tail_len);
+  if (st == WF_OK && (long)p.total_frames > e->cap_frames)
+    st = fail(e, WF_ERR_CAPACITY, "more than %ld frames", e->cap_frames);
   if (st != WF_OK) return st;
   if (cu_out)
     for (int i = 0; i <= B; ++i) cu_out[i] = e->meta_host[slot][p.ml.tok_off + i];
@@ -362,7 +367,7 @@ wf_status encode_impl(wf_encoder* e, const float* audio, const float* mel, const
       Prof pr(e, 0, s);
       launch_fill_seq_max(e->seq_max, B, s);
       launch_frontend(audio, meta, p.ml, B, p.n_fe_tiles, e->dft_basis, e->mel_fb_t, c.n_mel, e->logmel,
-                      e->seq_max, s);
+                      e->seq_max, tail, tail_len, s);
     }
     {
       Prof pr(e, 1, s);
@@ -470,7 +475,8 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
   }
   // workspace
   const size_t mt = (size_t)c.max_tokens;
-  WF_TRY(dev_alloc<float>(e, &e->logmel, (size_t)(c.max_samples / kHop + 1) * c.n_mel));
+  e->cap_frames = c.max_samples / kHop + (long)c.max_batch * (kMaxTailSamples / kHop) + 1;
+  WF_TRY(dev_alloc<float>(e, &e->logmel, (size_t)e->cap_frames * c.n_mel));
   WF_TRY(dev_alloc<int>(e, &e->seq_max, c.max_batch));
   WF_TRY(dev_alloc_bytes(e, &e->zp_alloc, (size_t)(e->cap_prows + 4) * e->mel_ld * e->esz, true));
   WF_TRY(dev_alloc_bytes(e, &e->c1p, (size_t)(e->cap_prows + 4) * d * e->esz, true));
@@ -570,7 +576,7 @@ wf_status wf_logmel(wf_encoder* e, const float* audio, const long* lengths, int 
     Prof pr(e, 0, s);
     launch_fill_seq_max(e->seq_max, B, s);
     launch_frontend(audio, meta, p.ml, B, p.n_fe_tiles, e->dft_basis, e->mel_fb_t, e->cfg.n_mel, e->logmel,
-                    e->seq_max, s);
+                    e->seq_max, nullptr, 0, s);
   }
   {
     Prof pr(e, 1, s);
@@ -584,6 +590,18 @@ wf_status wf_logmel(wf_encoder* e, const float* audio, const long* lengths, int 
 wf_status wf_encode(wf_encoder* e, const float* audio, const long* lengths, int B, const float* hush_mel,
                     void* hidden_out, int* cu_seqlens_out, void* stream) {
   return encode_impl(e, audio, nullptr, lengths, B, hush_mel, hidden_out, cu_seqlens_out, (cudaStream_t)stream);
+}
+
+wf_status wf_encode_raw_hush(wf_encoder* e, const float* audio, const long* lengths, int B,
+                             const float* hush_audio, int hush_samples, void* hidden_out, int* cu_seqlens_out,
+                             void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  if (e->cfg.hush_frames != 0)
+    return fail(e, WF_ERR_INVALID_ARG, "wf_encode_raw_hush needs an encoder created with hush_frames == 0");
+  if (hush_samples < 0 || hush_samples > kMaxTailSamples || (hush_samples > 0 && !hush_audio))
+    return fail(e, WF_ERR_INVALID_ARG, "hush_samples must be in [0, %d] with a non-NULL hush_audio", kMaxTailSamples);
+  return encode_impl(e, audio, nullptr, lengths, B, nullptr, hidden_out, cu_seqlens_out, (cudaStream_t)stream,
+                     hush_audio, hush_samples);
 }
 
 wf_status wf_encode_mel(wf_encoder* e, const float* mel, const long* frames, int B, const float* hush_mel,

@@ -74,7 +74,7 @@ constexpr int kPStride = 204;
 __global__ void __launch_bounds__(256) frontend_kernel(
     const float* __restrict__ audio, const int* __restrict__ meta, MetaLayout ml, int B,
     const float* __restrict__ basis, const float* __restrict__ fbt, int n_mel,
-    float* __restrict__ logmel, int* __restrict__ seq_max) {
+    float* __restrict__ logmel, int* __restrict__ seq_max, const float* __restrict__ tail, int tail_len) {
   extern __shared__ __align__(16) float smem[];
   float* e_s = smem;                       // [64][200]
   float* o_s = smem + kFeFrames * kFold;   // [64][200]
@@ -91,7 +91,8 @@ __global__ void __launch_bounds__(256) frontend_kernel(
   const int t0 = (tile - tile_off[seq]) * kFeFrames;
   const int T = meta[ml.frames + seq];
   const int s0 = meta[ml.sample_off + seq];
-  const int L = meta[ml.sample_off + seq + 1] - s0;
+  const int L_audio = meta[ml.sample_off + seq + 1] - s0;
+  const int L = L_audio + tail_len;  // the buffer followed by the raw-audio hush word, if any
   const float* x = audio + s0;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -106,9 +107,9 @@ __global__ void __launch_bounds__(256) frontend_kernel(
       if (ia >= L) ia = 2 * (L - 1) - ia;
       if (ib < 0) ib = -ib;
       if (ib >= L) ib = 2 * (L - 1) - ib;
-      float a = x[ia];
+      float a = ia < L_audio ? x[ia] : tail[ia - L_audio];
       if (n == kFold) { e = a; }
-      else { float b = x[ib]; e = a + b; o = a - b; }
+      else { float b = ib < L_audio ? x[ib] : tail[ib - L_audio]; e = a + b; o = a - b; }
     }
     e_s[idx] = e;
     o_s[idx] = o;
@@ -206,7 +207,7 @@ __global__ void __launch_bounds__(256) frontend_kernel(
 
 void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, int n_tiles,
                      const float* dft_basis, const float* mel_fb_t, int n_mel, float* logmel,
-                     int* seq_max, cudaStream_t s) {
+                     int* seq_max, const float* tail, int tail_len, cudaStream_t s) {
   const int smem = (kFeFrames * kPStride > 2 * kFeFrames * kFold ? kFeFrames * kPStride : 2 * kFeFrames * kFold) *
                    (int)sizeof(float);  // 102,400 B
   static bool configured = false;
@@ -216,7 +217,7 @@ void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, 
   }
   if (n_tiles > 0)
     frontend_kernel<<<n_tiles, 256, smem, s>>>(audio, meta, ml, B, dft_basis, mel_fb_t, n_mel, logmel,
-                                                seq_max);
+                                                seq_max, tail, tail_len);
 }
 
 // ---------------------------------------------------------------------------------------------

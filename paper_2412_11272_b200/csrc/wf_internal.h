@@ -57,6 +57,7 @@ void launch_build_tables(float* dft_basis /*[2][kFold][kBasisCols]*/, float* pe,
 void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, int n_tiles,
                      const float* dft_basis, const float* mel_fb_t /*[201][n_mel]*/, int n_mel,
                      float* logmel /*[sum T, n_mel]*/, int* seq_max /*[B] ordered ints*/,
+                     const float* tail /*tail_len samples that follow EVERY buffer, or NULL*/, int tail_len,
                      cudaStream_t s);
 // mode 0: packed normalised mel (float) for wf_logmel; mode 1: padded-row layout + hush rows.
 void launch_normalise(const float* logmel, const int* seq_max, const float* mel_in,

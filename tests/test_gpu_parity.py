@@ -126,6 +126,44 @@ def test_encode_mel_entry_and_raw_audio_level_hush():
     enc.close()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_raw_audio_level_hush_fused_in_front_end(dtype):
+    """wf_encode_raw_hush reads the hush samples in place (no concatenated copy) and must equal the
+    oracle's raw-audio-level variant, including frames that straddle the junction."""
+    shape = _small(dtype, d_model=256, n_head=4, d_mlp=512)
+    W = I.encoder_weights(12, shape)
+    lengths = [160 * 40, 160 * 7 + 93, 401, 160 * 130 + 159]        # junctions on and off the frame grid
+    batch = I.batch_from_lengths(13, lengths)
+    h = I.hush_audio(13)                                             # 8000 samples
+    enc = make_encoder(shape, W, 4, 512, int(sum(lengths)), hush_frames=0)
+    out, cu = enc.wf_encode_raw_hush(_dev(batch.audio), batch.lengths, _dev(h))
+    enc.wf_check()
+    got = to_np(out)
+    F = I.mel_filterbank(80)
+    assert list(np.diff(cu)) == [((n + 8000) // 160 + 1) // 2 for n in lengths]
+    for i, x in enumerate(batch.sequences()):
+        ref = O.encode_sequence(x, F, h, W, shape.n_layer, shape.n_head, hush_level="audio")
+        g = got[cu[i]:cu[i + 1]]
+        if dtype == "f32":
+            assert np.max(np.abs(g - ref)) <= F32_TOL, i
+        else:
+            _check_bf16(g, ref)
+    # the fused path equals running on caller-concatenated samples
+    cat = np.concatenate([np.concatenate([x, h]) for x in batch.sequences()]).astype(np.float32)
+    out2, cu2 = enc2_encode(shape, W, cat, [n + 8000 for n in lengths])
+    assert list(cu2) == list(cu) and np.max(np.abs(to_np(out2) - got)) <= (1e-5 if dtype == "f32" else 2e-2)
+    enc.close()
+
+
+def enc2_encode(shape, W, audio, lengths):
+    enc = make_encoder(shape, W, len(lengths), 1024, int(sum(lengths)), hush_frames=0)
+    out, cu = enc.wf_encode(_dev(audio), lengths, None)
+    enc.wf_check()
+    res = (out.clone(), cu)
+    enc.close()
+    return res
+
+
 # ------------------------------------------------------------------------------ bf16 components
 
 @pytest.mark.parametrize("M,N,K", [(300, 384, 240), (1000, 1536, 512), (129, 256, 64), (4097, 1280, 1280),
