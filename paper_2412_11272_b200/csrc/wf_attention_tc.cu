@@ -340,10 +340,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
               tmem_st_wait();
             }
           }
-          // the probability buffer of this step was last read by the P V of two steps ago
-          if (j >= 2) {
-            if (!wait_warp(o_full(t, g & 1u), ((g - 2) >> 1) & 1u)) { ok = false; break; }
-          }
+          // The probability buffer of this step was last read by the P V of two steps ago.  That
+          // product was issued, by the same thread, before the S of this step, and the commit
+          // behind S tracks every earlier MMA of that thread: having seen s_full, it has landed.
           float rs = 0.f, rs1 = 0.f;
           const uint32_t ta_p = ta_s + 96 + 48 * (g & 1u);
 #pragma unroll
@@ -365,15 +364,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
           }
           l_run += rs + rs1;
           tmem_st_wait();
-        } else if (j >= 2) {
-          if (!wait_warp(o_full(t, g & 1u), ((g - 2) >> 1) & 1u)) { ok = false; break; }
         }
         tc_fence_before();
         mbar_arrive(p_full(t, g & 1u));
         ++g;
       }
       if (!ok) break;
-      // drain the last two products (each barrier phase is waited for exactly in order)
+      // drain the last two products (earlier phases of these barriers completed before the
+      // s_full waits above returned, so the parities below are unambiguous)
       if (w.n_kv >= 2) {
         if (!wait_warp(o_full(t, (g - 2) & 1u), ((g - 2) >> 1) & 1u)) { ok = false; break; }
       }
