@@ -165,6 +165,25 @@ wf_status wf_gemm_bf16(wf_encoder *enc, const void *A, const void *W, const floa
 wf_status wf_attention(wf_encoder *enc, const void *qkv, const int *cu_seqlens, int B, void *out,
                        void *stream);
 
+/* Beam-pruning state machine (Sec. 4.2.2, "New design in beam pruning"): host-side integer logic
+ * that tells a beam-search decoder which beam size to use in its next round, given the top-1
+ * token of the current round and the previous round's transcript as a reference.  Decoding
+ * starts with beam 1; the first comparable top-1 token is searched through the reference
+ * (alignment; the aligned token counts as matched); afterwards a comparable token must equal the
+ * next reference token; tokens flagged special (punctuation, timestamps, other special ids) are
+ * never compared and leave the state unchanged; a failed search, a mismatch or an exhausted
+ * reference restores `full_beam` until the session ends.
+ *   reference   host  n_reference token ids (copied);  is_special  host  vocab_size flags (copied)
+ *   wf_beam_pruner_step returns the beam size for the NEXT round, or -1 on a bad argument. */
+typedef struct wf_beam_pruner wf_beam_pruner;
+wf_status wf_beam_pruner_create(const int *reference, int n_reference, const unsigned char *is_special,
+                                int vocab_size, int full_beam, wf_beam_pruner **out);
+int wf_beam_pruner_step(wf_beam_pruner *p, int top1_token);
+/* reference_index: next position to compare with (-1 before alignment); any pointer may be NULL */
+wf_status wf_beam_pruner_state(const wf_beam_pruner *p, long *reference_index, int *fallen_back,
+                               long *rounds, long *rounds_at_one);
+wf_status wf_beam_pruner_destroy(wf_beam_pruner *p);
+
 /* wf_attention_f32_static: wf_attention for float32 activations without an encoder handle and
  * without any allocation (the paper has no counterpart; this exists for integration only).
  * It is meant for callers that cannot call cudaMalloc: code running inside a process whose

@@ -54,7 +54,8 @@ _PER_LAYER = ("ln1_g", "ln1_b", "wq", "bq", "wk", "wv", "bv", "wo", "bo", "ln2_g
 
 EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_raw_hush", "wf_encode_mel", "wf_encode_host", "wf_check",
            "wf_encoder_destroy", "wf_last_error", "wf_profile_enable", "wf_profile_read",
-           "wf_gemm_bf16", "wf_attention", "wf_attention_f32_static")
+           "wf_gemm_bf16", "wf_attention", "wf_attention_f32_static",
+           "wf_beam_pruner_create", "wf_beam_pruner_step", "wf_beam_pruner_state", "wf_beam_pruner_destroy")
 
 _lib = None
 
@@ -83,6 +84,10 @@ def load_library() -> C.CDLL:
     lib.wf_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, C.c_long, C.c_int, C.c_int, C.c_int, vp]
     lib.wf_attention.argtypes = [vp, vp, ip, C.c_int, vp, vp]
     lib.wf_attention_f32_static.argtypes = [vp, ip, C.c_int, C.c_int, vp, vp]
+    lib.wf_beam_pruner_create.argtypes = [ip, C.c_int, C.POINTER(C.c_ubyte), C.c_int, C.c_int, C.POINTER(vp)]
+    lib.wf_beam_pruner_step.argtypes = [vp, C.c_int]
+    lib.wf_beam_pruner_state.argtypes = [vp, lp, ip, lp, lp]
+    lib.wf_beam_pruner_destroy.argtypes = [vp]
     for name in EXPORTS:
         if name != "wf_last_error":
             getattr(lib, name).restype = C.c_int
@@ -276,3 +281,42 @@ def wf_attention_f32_static(qkv: torch.Tensor, cu_seqlens, d_model: int, out: to
     if st != 0:
         raise WfError(st, "wf_attention_f32_static rejected its arguments or a CUDA call failed")
     return out
+
+
+class BeamPruner:
+    """Marshals the host-side beam-pruning state machine (wf_beam_pruner_*)."""
+
+    def __init__(self, reference, is_special, full_beam: int = 5):
+        self.lib = load_library()
+        ref = np.ascontiguousarray(np.asarray(reference, dtype=np.int32))
+        flags = np.ascontiguousarray(np.asarray(is_special, dtype=np.uint8))
+        h = C.c_void_p()
+        st = self.lib.wf_beam_pruner_create(ref.ctypes.data_as(C.POINTER(C.c_int)), len(ref),
+                                            flags.ctypes.data_as(C.POINTER(C.c_ubyte)), len(flags), int(full_beam),
+                                            C.byref(h))
+        if st != 0:
+            raise WfError(st, "wf_beam_pruner_create rejected its arguments")
+        self.handle = h
+
+    def step(self, top1: int) -> int:
+        r = self.lib.wf_beam_pruner_step(self.handle, int(top1))
+        if r < 0:
+            raise WfError(1, "wf_beam_pruner_step: token id outside the vocabulary")
+        return r
+
+    def state(self):
+        idx, rounds, ones, fb = C.c_long(), C.c_long(), C.c_long(), C.c_int()
+        self.lib.wf_beam_pruner_state(self.handle, C.byref(idx), C.byref(fb), C.byref(rounds), C.byref(ones))
+        return {"reference_index": idx.value, "fallen_back": bool(fb.value), "rounds": rounds.value,
+                "rounds_at_one": ones.value}
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.wf_beam_pruner_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
