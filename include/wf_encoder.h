@@ -165,6 +165,20 @@ wf_status wf_gemm_bf16(wf_encoder *enc, const void *A, const void *W, const floa
 wf_status wf_attention(wf_encoder *enc, const void *qkv, const int *cu_seqlens, int B, void *out,
                        void *stream);
 
+/* wf_dtw: dynamic time warping of B token-by-frame cost matrices (token timestamping from the
+ * decoder's cross-attention, Sec. 3.2 "Workload mapping" and Sec. 4.3.2, which name DTW and give
+ * no further detail: this is the classic recurrence D[i,j] = C[i,j] + min(D[i-1,j-1], D[i-1,j],
+ * D[i,j-1]) with the path traced back from the last cell; float32; ties prefer the diagonal,
+ * then the token step, then the frame step).
+ *   cost         dev  float32, problem b is a row-major [n_tokens[b], n_frames[b]] matrix, the
+ *                     problems back to back
+ *   n_tokens, n_frames  host  B sizes (tokens <= 16384; fewer than 2^31 cells in total)
+ *   trace_ws     dev  scratch, one byte per cost cell (caller-owned)
+ *   token_start  dev  int32, sum of n_tokens entries: first frame of every token on the path
+ *   total_cost   dev  float32 [B]: D at the last cell */
+wf_status wf_dtw(wf_encoder *enc, const float *cost, const int *n_tokens, const int *n_frames, int B,
+                 unsigned char *trace_ws, int *token_start, float *total_cost, void *stream);
+
 /* Beam-pruning state machine (Sec. 4.2.2, "New design in beam pruning"): host-side integer logic
  * that tells a beam-search decoder which beam size to use in its next round, given the top-1
  * token of the current round and the previous round's transcript as a reference.  Decoding

@@ -54,7 +54,7 @@ _PER_LAYER = ("ln1_g", "ln1_b", "wq", "bq", "wk", "wv", "bv", "wo", "bo", "ln2_g
 
 EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_raw_hush", "wf_encode_mel", "wf_encode_host", "wf_check",
            "wf_encoder_destroy", "wf_last_error", "wf_profile_enable", "wf_profile_read",
-           "wf_gemm_bf16", "wf_attention", "wf_attention_f32_static",
+           "wf_gemm_bf16", "wf_attention", "wf_dtw", "wf_attention_f32_static",
            "wf_beam_pruner_create", "wf_beam_pruner_step", "wf_beam_pruner_state", "wf_beam_pruner_destroy")
 
 _lib = None
@@ -83,6 +83,7 @@ def load_library() -> C.CDLL:
     lib.wf_profile_read.argtypes = [vp, lp, C.POINTER(C.c_double)]
     lib.wf_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, C.c_long, C.c_int, C.c_int, C.c_int, vp]
     lib.wf_attention.argtypes = [vp, vp, ip, C.c_int, vp, vp]
+    lib.wf_dtw.argtypes = [vp, vp, ip, ip, C.c_int, vp, vp, vp, vp]
     lib.wf_attention_f32_static.argtypes = [vp, ip, C.c_int, C.c_int, vp, vp]
     lib.wf_beam_pruner_create.argtypes = [ip, C.c_int, C.POINTER(C.c_ubyte), C.c_int, C.c_int, C.POINTER(vp)]
     lib.wf_beam_pruner_step.argtypes = [vp, C.c_int]
@@ -262,6 +263,21 @@ class Encoder:
         self._check(self.lib.wf_gemm_bf16(self.handle, A.data_ptr(), W.data_ptr(), bias.data_ptr(),
                                           C_out.data_ptr(), M, N, K, mode, _stream_ptr(stream)))
         return C_out
+
+    def wf_dtw(self, cost: torch.Tensor, n_tokens, n_frames, stream=None):
+        """cost: float32 CUDA tensor holding the B matrices back to back.  Returns
+        (token_start int32 [sum n_tokens], total_cost float32 [B]) as CUDA tensors."""
+        nt = np.ascontiguousarray(np.asarray(n_tokens, dtype=np.int32))
+        nf = np.ascontiguousarray(np.asarray(n_frames, dtype=np.int32))
+        B = len(nt)
+        cells = int((nt.astype(np.int64) * nf).sum())
+        trace = torch.empty(max(cells, 1), dtype=torch.uint8, device=cost.device)
+        start = torch.empty(max(int(nt.sum()), 1), dtype=torch.int32, device=cost.device)
+        total = torch.empty(max(B, 1), dtype=torch.float32, device=cost.device)
+        ip = C.POINTER(C.c_int)
+        self._check(self.lib.wf_dtw(self.handle, cost.data_ptr(), nt.ctypes.data_as(ip), nf.ctypes.data_as(ip), B,
+                                    trace.data_ptr(), start.data_ptr(), total.data_ptr(), _stream_ptr(stream)))
+        return start[:int(nt.sum())], total[:B]
 
     def wf_attention(self, qkv: torch.Tensor, cu_seqlens, stream=None):
         cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))

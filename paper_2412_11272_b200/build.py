@@ -17,7 +17,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libwf_encoder.so")
-SOURCES = ["wf_api.cu", "wf_frontend.cu", "wf_simt.cu", "wf_gemm_tcgen05.cu", "wf_attention_tc.cu", "wf_static.cu", "wf_beam.cu"]
+SOURCES = ["wf_api.cu", "wf_frontend.cu", "wf_simt.cu", "wf_gemm_tcgen05.cu", "wf_attention_tc.cu", "wf_static.cu", "wf_beam.cu", "wf_dtw.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

@@ -686,6 +686,41 @@ wf_status wf_gemm_bf16(wf_encoder* e, const void* A, const void* W, const float*
   return WF_OK;
 }
 
+wf_status wf_dtw(wf_encoder* e, const float* cost, const int* n_tokens, const int* n_frames, int B,
+                 unsigned char* trace_ws, int* token_start, float* total_cost, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (B < 0 || (B > 0 && (!cost || !n_tokens || !n_frames || !trace_ws || !token_start || !total_cost)))
+    return fail(e, WF_ERR_INVALID_ARG, "wf_dtw: NULL argument");
+  if (B == 0) return WF_OK;
+  if (4 * B > e->meta_cap) return fail(e, WF_ERR_CAPACITY, "wf_dtw: batch %d exceeds the metadata capacity", B);
+  int slot;
+  wf_status st = ring_acquire(e, &slot);
+  if (st != WF_OK) return st;
+  int* hm = e->meta_host[slot];
+  long cells = 0, toks = 0;
+  int max_tok = 0;
+  for (int b = 0; b < B; ++b) {
+    if (n_tokens[b] < 1 || n_frames[b] < 1 || n_tokens[b] > 16384)
+      return fail(e, WF_ERR_INVALID_ARG, "wf_dtw: problem %d has %d tokens x %d frames", b, n_tokens[b], n_frames[b]);
+    if (cells + (long)n_tokens[b] * n_frames[b] >= (1L << 31))
+      return fail(e, WF_ERR_CAPACITY, "wf_dtw: more than 2^31 cells in one call");
+    hm[4 * b] = (int)cells;
+    hm[4 * b + 1] = n_tokens[b];
+    hm[4 * b + 2] = n_frames[b];
+    hm[4 * b + 3] = (int)toks;
+    cells += (long)n_tokens[b] * n_frames[b];
+    toks += n_tokens[b];
+    max_tok = std::max(max_tok, n_tokens[b]);
+  }
+  Plan p{};
+  p.ml.total = 4 * B;
+  st = ring_upload(e, slot, p, s);
+  if (st != WF_OK) return st;
+  WF_CUDA(e, launch_dtw(cost, e->meta_dev[slot], B, max_tok, trace_ws, token_start, total_cost, s));
+  return ring_release(e, slot, s);
+}
+
 wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, int B, void* out, void* stream) {
   if (!e) return WF_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;

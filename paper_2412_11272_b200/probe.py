@@ -42,7 +42,7 @@ def _component_encoder(d_model=128, n_head=2, max_batch=1, max_tokens=64):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["gemm", "attention", "encode", "logmel", "config"])
+    ap.add_argument("what", choices=["gemm", "attention", "encode", "logmel", "config", "dtw"])
     ap.add_argument("--name", default="base")
     ap.add_argument("--M", type=int, default=16384)
     ap.add_argument("--N", type=int, default=3840)
@@ -73,6 +73,17 @@ def main():
         ms = _time(lambda: enc.wf_attention(qkv, cu), a.iters)
         enc.wf_check()
         out.update(n=a.n, batch=a.batch, d_model=d, ms=ms, tflops=4.0 * a.batch * a.n * a.n * d / ms / 1e9)
+    elif a.what == "dtw":
+        # --batch problems of --n tokens x (5 * --n) frames (150 tokens x 750 frames by default)
+        n_tok, n_frm = (a.n if a.n != 775 else 150), 5 * (a.n if a.n != 775 else 150)
+        enc = _component_encoder(128, 2, max(a.batch, 1), 64)
+        cost = torch.as_tensor(np.concatenate([I.dtw_cost(0, b, n_tok, n_frm).reshape(-1) for b in range(a.batch)])).cuda()
+        nt, nf = [n_tok] * a.batch, [n_frm] * a.batch
+        ms = _time(lambda: enc.wf_dtw(cost, nt, nf), a.iters)
+        enc.wf_check()
+        cells = a.batch * n_tok * n_frm
+        out.update(batch=a.batch, n_tok=n_tok, n_frm=n_frm, ms=ms, gcells_per_s=cells / ms / 1e6,
+                   gbs=cells * 5.0 / ms / 1e6, sequential_steps=n_tok + n_frm - 1)
     elif a.what == "config":
         # one named configuration end to end (device-resident inputs), per-call times with CUDA events
         base = a.name.split("-")[0]
