@@ -700,6 +700,7 @@ wf_status wf_dtw(wf_encoder* e, const float* cost, const int* n_tokens, const in
   int* hm = e->meta_host[slot];
   long cells = 0, toks = 0;
   int max_tok = 0;
+  long max_cells = 0;
   for (int b = 0; b < B; ++b) {
     if (n_tokens[b] < 1 || n_frames[b] < 1 || n_tokens[b] > 16384)
       return fail(e, WF_ERR_INVALID_ARG, "wf_dtw: problem %d has %d tokens x %d frames", b, n_tokens[b], n_frames[b]);
@@ -712,12 +713,13 @@ wf_status wf_dtw(wf_encoder* e, const float* cost, const int* n_tokens, const in
     cells += (long)n_tokens[b] * n_frames[b];
     toks += n_tokens[b];
     max_tok = std::max(max_tok, n_tokens[b]);
+    max_cells = std::max(max_cells, (long)n_tokens[b] * n_frames[b]);
   }
   Plan p{};
   p.ml.total = 4 * B;
   st = ring_upload(e, slot, p, s);
   if (st != WF_OK) return st;
-  WF_CUDA(e, launch_dtw(cost, e->meta_dev[slot], B, max_tok, trace_ws, token_start, total_cost, s));
+  WF_CUDA(e, launch_dtw(cost, e->meta_dev[slot], B, max_tok, max_cells, trace_ws, token_start, total_cost, s));
   return ring_release(e, slot, s);
 }
 

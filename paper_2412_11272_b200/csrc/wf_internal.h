@@ -113,7 +113,8 @@ void launch_attention_bf16(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv
 
 // ---- dynamic time warping (wf_dtw.cu); meta holds 4 ints per problem:
 // cost offset in cells, tokens, frames, offset into token_start
-cudaError_t launch_dtw(const float* cost, const int* meta, int B, int max_tok, unsigned char* trace,
+cudaError_t launch_dtw(const float* cost, const int* meta, int B, int max_tok, long max_cells,
+                       unsigned char* trace,
                        int* token_start, float* total_cost, cudaStream_t s);
 
 }  // namespace wf

@@ -302,18 +302,21 @@ def test_dtw_matches_oracle_bit_for_bit():
     from oracle import dtw_oracle
     shape = _small("f32", n_layer=0)
     enc = make_encoder(shape, I.encoder_weights(0, shape), 8, 64, 1000)
-    sizes = [(40, 300), (1, 17), (23, 1), (150, 775), (300, 97), (7, 7)]     # ragged, degenerate, wide, tall
-    costs = [I.dtw_cost(4, b, n, m) for b, (n, m) in enumerate(sizes)]
-    packed = np.concatenate([c.reshape(-1) for c in costs])
-    start, total = enc.wf_dtw(_dev(packed), [n for n, _ in sizes], [m for _, m in sizes])
-    enc.wf_check()
-    start, total = start.cpu().numpy(), total.cpu().numpy()
-    off = 0
-    for b, c in enumerate(costs):
-        t_ref, _, s_ref = dtw_oracle.dtw(c)
-        assert total[b] == t_ref                                   # same float32 additions, same order
-        assert np.array_equal(start[off:off + len(s_ref)], s_ref), b
-        off += len(s_ref)
+    # first batch: ragged, degenerate, wide, tall, all small enough for the arg-min bytes to stay in
+    # shared memory; second batch: a problem too large for that (bytes go to the workspace) and one
+    # with more tokens than threads (several cells per thread and anti-diagonal)
+    for batch in ([(40, 300), (1, 17), (23, 1), (150, 775), (300, 97), (7, 7)], [(300, 900), (5, 9), (600, 300)]):
+        costs = [I.dtw_cost(4, b, n, m) for b, (n, m) in enumerate(batch)]
+        packed = np.concatenate([c.reshape(-1) for c in costs])
+        start, total = enc.wf_dtw(_dev(packed), [n for n, _ in batch], [m for _, m in batch])
+        enc.wf_check()
+        start, total = start.cpu().numpy(), total.cpu().numpy()
+        off = 0
+        for b, c in enumerate(costs):
+            t_ref, _, s_ref = dtw_oracle.dtw(c)
+            assert total[b] == t_ref                               # same float32 additions, same order
+            assert np.array_equal(start[off:off + len(s_ref)], s_ref), (batch, b)
+            off += len(s_ref)
     enc.close()
 
 
