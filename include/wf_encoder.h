@@ -165,6 +165,21 @@ wf_status wf_gemm_bf16(wf_encoder *enc, const void *A, const void *W, const floa
 wf_status wf_attention(wf_encoder *enc, const void *qkv, const int *cu_seqlens, int B, void *out,
                        void *stream);
 
+/* wf_cross_kv: the cross-attention key and value projections of the encoder's output for every
+ * decoder layer in one GEMM, kv = hidden W_kv^T + b_kv: the first thing prompt prefill (Sec. 3.2
+ * "Operations", Sec. 4.3.2) needs from the encoding stage, and the same for every later decoding
+ * round on this buffer.  Runs on the encoder's path (tcgen05 for WF_BF16, float32 SIMT else).
+ *   hidden  dev  [M, d_model]                   path dtype (what wf_encode wrote)
+ *   W_kv    dev  [n_dec_layers * 2 d_model, d_model] path dtype, row-major: rows
+ *                [2 l d, 2 l d + d) are layer l's key weight, the next d rows its value weight
+ *   b_kv    dev  float32 [n_dec_layers * 2 d_model] (the architecture's key projection has no
+ *                bias: those slices are zero)
+ *   kv      dev  [M, n_dec_layers * 2 d_model]  path dtype; layer l's keys are columns
+ *                [2 l d, 2 l d + d) of every row, its values the next d columns
+ * On the bf16 path all pointers must be 16-byte aligned. */
+wf_status wf_cross_kv(wf_encoder *enc, const void *hidden, const void *W_kv, const float *b_kv,
+                      long M, int n_dec_layers, void *kv, void *stream);
+
 /* wf_dtw: dynamic time warping of B token-by-frame cost matrices (token timestamping from the
  * decoder's cross-attention, Sec. 3.2 "Workload mapping" and Sec. 4.3.2, which name DTW and give
  * no further detail: this is the classic recurrence D[i,j] = C[i,j] + min(D[i-1,j-1], D[i-1,j],

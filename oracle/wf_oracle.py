@@ -233,3 +233,14 @@ def encode_batch(seqs, mel_fb, hush, weights, n_layer, n_head, hush_level="mel")
     d = np.asarray(weights["lnp_g"]).shape[0]
     packed = np.concatenate(outs, axis=0) if outs else np.zeros((0, d))
     return packed, cu
+
+
+def cross_kv(hidden, wk, wv, bv):
+    """Cross-attention keys and values the decoder's layers read from the encoder output
+    (the step right after the encoding stage, Sec. 3.2 "Operations"): for decoder layer l,
+    K_l = hidden wk[l]^T (no bias) and V_l = hidden wv[l]^T + bv[l].
+    hidden [n, d]; wk, wv [L, d, d] as [out, in]; bv [L, d].  Returns (K, V), each [L, n, d]."""
+    h = np.asarray(hidden, dtype=np.float64)
+    K = np.stack([h @ np.asarray(w, dtype=np.float64).T for w in wk])
+    V = np.stack([h @ np.asarray(w, dtype=np.float64).T + np.asarray(b, dtype=np.float64) for w, b in zip(wv, bv)])
+    return K, V

@@ -54,7 +54,7 @@ _PER_LAYER = ("ln1_g", "ln1_b", "wq", "bq", "wk", "wv", "bv", "wo", "bo", "ln2_g
 
 EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_raw_hush", "wf_encode_mel", "wf_encode_host", "wf_check",
            "wf_encoder_destroy", "wf_last_error", "wf_profile_enable", "wf_profile_read",
-           "wf_gemm_bf16", "wf_attention", "wf_dtw", "wf_attention_f32_static",
+           "wf_gemm_bf16", "wf_attention", "wf_cross_kv", "wf_dtw", "wf_attention_f32_static",
            "wf_beam_pruner_create", "wf_beam_pruner_step", "wf_beam_pruner_state", "wf_beam_pruner_destroy")
 
 _lib = None
@@ -83,6 +83,7 @@ def load_library() -> C.CDLL:
     lib.wf_profile_read.argtypes = [vp, lp, C.POINTER(C.c_double)]
     lib.wf_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, C.c_long, C.c_int, C.c_int, C.c_int, vp]
     lib.wf_attention.argtypes = [vp, vp, ip, C.c_int, vp, vp]
+    lib.wf_cross_kv.argtypes = [vp, vp, vp, vp, C.c_long, C.c_int, vp, vp]
     lib.wf_dtw.argtypes = [vp, vp, ip, ip, C.c_int, vp, vp, vp, vp]
     lib.wf_attention_f32_static.argtypes = [vp, ip, C.c_int, C.c_int, vp, vp]
     lib.wf_beam_pruner_create.argtypes = [ip, C.c_int, C.POINTER(C.c_ubyte), C.c_int, C.c_int, C.POINTER(vp)]
@@ -263,6 +264,16 @@ class Encoder:
         self._check(self.lib.wf_gemm_bf16(self.handle, A.data_ptr(), W.data_ptr(), bias.data_ptr(),
                                           C_out.data_ptr(), M, N, K, mode, _stream_ptr(stream)))
         return C_out
+
+    def wf_cross_kv(self, hidden: torch.Tensor, W_kv: torch.Tensor, b_kv: torch.Tensor, kv_out=None, stream=None):
+        """hidden [M, d], W_kv [n_dec * 2 d, d] (path dtype), b_kv float32 [n_dec * 2 d] -> kv [M, n_dec * 2 d]."""
+        M, d = hidden.shape
+        n_dec = W_kv.shape[0] // (2 * d)
+        if kv_out is None:
+            kv_out = torch.empty((M, W_kv.shape[0]), dtype=hidden.dtype, device=hidden.device)
+        self._check(self.lib.wf_cross_kv(self.handle, hidden.data_ptr(), W_kv.data_ptr(), b_kv.data_ptr(), M, n_dec,
+                                         kv_out.data_ptr(), _stream_ptr(stream)))
+        return kv_out
 
     def wf_dtw(self, cost: torch.Tensor, n_tokens, n_frames, stream=None):
         """cost: float32 CUDA tensor holding the B matrices back to back.  Returns

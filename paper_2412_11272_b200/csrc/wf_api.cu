@@ -686,6 +686,35 @@ wf_status wf_gemm_bf16(wf_encoder* e, const void* A, const void* W, const float*
   return WF_OK;
 }
 
+wf_status wf_cross_kv(wf_encoder* e, const void* hidden, const void* W_kv, const float* b_kv, long M,
+                      int n_dec_layers, void* kv, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  const int d = e->cfg.d_model;
+  if (M < 0 || n_dec_layers < 1 || (long)n_dec_layers * 2 * d > (1L << 30) || !W_kv || !b_kv ||
+      (M > 0 && (!hidden || !kv)))
+    return fail(e, WF_ERR_INVALID_ARG, "wf_cross_kv: bad pointer or size");
+  if (M == 0) return WF_OK;
+  const int N = n_dec_layers * 2 * d;
+  EpiParams ep{};
+  ep.bias = b_kv;
+  ep.ldc = N;
+  ep.out = kv;
+  if (e->bf16) {
+    if (((uintptr_t)hidden & 15) || ((uintptr_t)W_kv & 15) || ((uintptr_t)kv & 15) || ((uintptr_t)b_kv & 15))
+      return fail(e, WF_ERR_INVALID_ARG, "wf_cross_kv: pointers must be 16-byte aligned");
+    CUtensorMap ta, tb, tc;
+    if (!make_tmap_bf16(e->tma, &ta, hidden, d, M, d, 128) ||
+        !make_tmap_bf16(e->tma, &tb, W_kv, d, N, d, gemm_bf16_uses_pair() ? 128 : 256) ||
+        !make_tmap_out(e->tma, &tc, kv, 2, N, M))
+      return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
+    launch_gemm_bf16(ta, tb, tc, M, N, d, d, kEpiBias, ep, e->err_flag, e->num_sms, (cudaStream_t)stream);
+  } else {
+    launch_gemm_f32((const float*)hidden, d, (const float*)W_kv, d, M, N, d, kEpiBias, ep, (cudaStream_t)stream);
+  }
+  WF_CUDA(e, cudaGetLastError());
+  return WF_OK;
+}
+
 wf_status wf_dtw(wf_encoder* e, const float* cost, const int* n_tokens, const int* n_frames, int B,
                  unsigned char* trace_ws, int* token_start, float* total_cost, void* stream) {
   if (!e) return WF_ERR_INVALID_ARG;

@@ -4,6 +4,8 @@
     python -m paper_2412_11272_b200.probe attention --n 775 --batch 64
     python -m paper_2412_11272_b200.probe encode --shape large --seconds 3 --batch 16
     python -m paper_2412_11272_b200.probe logmel --seconds 15 --batch 64
+    python -m paper_2412_11272_b200.probe dtw --batch 64 --n 150
+    python -m paper_2412_11272_b200.probe crosskv --M 49600 --layers 32
     python -m paper_2412_11272_b200.probe config --name small        (tiny, base, small, medium-padded, medium-hush, large)
 
 Each command warms up, times ``--iters`` launches with CUDA events on the launching stream and
@@ -42,7 +44,7 @@ def _component_encoder(d_model=128, n_head=2, max_batch=1, max_tokens=64):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["gemm", "attention", "encode", "logmel", "config", "dtw"])
+    ap.add_argument("what", choices=["gemm", "attention", "encode", "logmel", "config", "dtw", "crosskv"])
     ap.add_argument("--name", default="base")
     ap.add_argument("--M", type=int, default=16384)
     ap.add_argument("--N", type=int, default=3840)
@@ -53,6 +55,7 @@ def main():
     ap.add_argument("--d_model", type=int, default=1280)
     ap.add_argument("--shape", default="large")
     ap.add_argument("--seconds", type=float, default=3.0)
+    ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--iters", type=int, default=10)
     a = ap.parse_args()
     out = {"what": a.what}
@@ -73,6 +76,18 @@ def main():
         ms = _time(lambda: enc.wf_attention(qkv, cu), a.iters)
         enc.wf_check()
         out.update(n=a.n, batch=a.batch, d_model=d, ms=ms, tflops=4.0 * a.batch * a.n * a.n * d / ms / 1e9)
+    elif a.what == "crosskv":
+        # --M encoder tokens of width --d_model projected to the keys and values of --layers decoder layers
+        d, N = a.d_model, a.layers * 2 * a.d_model
+        enc = _component_encoder(d, d // 64)
+        hidden = torch.randn(a.M, d, device="cuda").to(torch.bfloat16)
+        W = (torch.randn(N, d, device="cuda") * 0.02).to(torch.bfloat16)
+        b = torch.zeros(N, device="cuda")
+        kv = torch.empty(a.M, N, device="cuda", dtype=torch.bfloat16)
+        ms = _time(lambda: enc.wf_cross_kv(hidden, W, b, kv), a.iters)
+        enc.wf_check()
+        out.update(M=a.M, d_model=d, layers=a.layers, ms=ms, tflops=2.0 * a.M * N * d / ms / 1e9,
+                   write_gbs=2.0 * a.M * N / ms / 1e6)
     elif a.what == "dtw":
         # --batch problems of --n tokens x (5 * --n) frames (150 tokens x 750 frames by default)
         n_tok, n_frm = (a.n if a.n != 775 else 150), 5 * (a.n if a.n != 775 else 150)

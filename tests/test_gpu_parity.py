@@ -195,6 +195,32 @@ def test_tcgen05_gemm_matches_fp64(M, N, K, mode):
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_cross_kv_projection_matches_oracle(dtype):
+    """Encoder output -> cross-attention keys/values of every decoder layer (one GEMM)."""
+    bf16 = dtype == "bf16"
+    shape = _small(dtype, n_layer=0, d_model=256 if bf16 else 128, n_head=4 if bf16 else 2, d_mlp=256)
+    d, L, M = shape.d_model, 3, 333                                   # ragged against the 128/256-row tiles
+    enc = make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000)
+    Wc = I.cross_kv_weights(11, d, L, bf16)
+    hidden = I.normal01(11, 6_100_000, M * d).astype(np.float32).reshape(M, d)
+    if bf16:
+        hidden = I.round_to_bf16(hidden)
+    K, V = O.cross_kv(hidden, Wc["wk"], Wc["wv"], Wc["bv"])
+    W_kv = np.concatenate([np.concatenate([Wc["wk"][l], Wc["wv"][l]]) for l in range(L)])      # [L * 2d, d]
+    b_kv = np.concatenate([np.concatenate([np.zeros(d, np.float32), Wc["bv"][l]]) for l in range(L)])
+    tdt = torch.bfloat16 if bf16 else torch.float32
+    kv = to_np(enc.wf_cross_kv(_dev(hidden, tdt), _dev(W_kv, tdt), _dev(b_kv)))
+    enc.wf_check()
+    assert kv.shape == (M, L * 2 * d)
+    for l in range(L):
+        for got, ref in ((kv[:, 2 * l * d:2 * l * d + d], K[l]), (kv[:, 2 * l * d + d:2 * (l + 1) * d], V[l])):
+            err = np.max(np.abs(got - ref))
+            assert err < (2.0 ** -8 * (np.max(np.abs(ref)) + 1e-3) if bf16 else 1e-5), (l, err)
+    assert enc.wf_cross_kv(_dev(hidden[:0], tdt), _dev(W_kv, tdt), _dev(b_kv)).shape[0] == 0   # empty
+    enc.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_varlen_attention_matches_oracle(dtype):
     shape = _small(dtype, n_layer=0, d_model=256, n_head=4, d_mlp=256)
     enc = make_encoder(shape, I.encoder_weights(0, shape), 8, 4096, 1000)

@@ -408,6 +408,27 @@ def test_pins_catch_planted_mistakes(monkeypatch):
 
 # ----- measurement sanity: hush vs 30 s padding (Sec. 2.2 and Sec. 6.3 quote 3-3.7x) ---------
 
+def test_cross_kv_hand_worked_and_linear():
+    """cross_kv against values worked by hand (a transposed weight, a bias on the keys or a
+    missing bias on the values would each change them) and against linearity."""
+    h = np.array([[1.0, 2.0], [0.0, -1.0], [3.0, 0.5]])
+    wk = np.array([[[1.0, 0.0], [2.0, -1.0]], [[0.0, 1.0], [1.0, 1.0]]])          # [L=2, out, in]
+    wv = np.array([[[0.5, 0.5], [0.0, 2.0]], [[-1.0, 0.0], [0.0, 0.0]]])
+    bv = np.array([[10.0, 20.0], [0.0, -5.0]])
+    K, V = O.cross_kv(h, wk, wv, bv)
+    assert K.shape == V.shape == (2, 3, 2)
+    # K_0[t] = (h0, 2 h0 - h1);  K_1[t] = (h1, h0 + h1)
+    assert np.array_equal(K[0], [[1.0, 0.0], [0.0, 1.0], [3.0, 5.5]])
+    assert np.array_equal(K[1], [[2.0, 3.0], [-1.0, -1.0], [0.5, 3.5]])
+    # V_0[t] = ((h0 + h1)/2 + 10, 2 h1 + 20);  V_1[t] = (-h0, -5)
+    assert np.array_equal(V[0], [[11.5, 24.0], [9.5, 18.0], [11.75, 21.0]])
+    assert np.array_equal(V[1], [[-1.0, -5.0], [0.0, -5.0], [-3.0, -5.0]])
+    K0, V0 = O.cross_kv(np.zeros_like(h), wk, wv, bv)                              # keys carry no bias
+    assert np.all(K0 == 0.0) and np.array_equal(V0[0], np.tile(bv[0], (3, 1)))
+    K2, V2 = O.cross_kv(2.0 * h, wk, wv, bv)
+    assert np.allclose(K2, 2.0 * K) and np.allclose(V2 - V0, 2.0 * (V - V0))
+
+
 def test_padding_vs_hush_flop_ratio():
     shape = I.SHAPES["medium"]
     clips = I.uniform_lengths(3, 256, 5, 25)                # the paper's clip lengths, 5-25 s
