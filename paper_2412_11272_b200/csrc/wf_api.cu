@@ -1,6 +1,7 @@
 // C ABI, host-side ragged planner and launch sequence of the encoder.
 #include <algorithm>
 #include <cstdarg>
+#include <cstdlib>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -9,6 +10,12 @@
 #include "wf_internal.h"
 
 using namespace wf;
+
+namespace wf {
+static int g_pdl = 1;
+int pdl_enabled() { return g_pdl; }
+void pdl_set(int on) { g_pdl = on; }
+}  // namespace wf
 
 namespace {
 constexpr int kRing = 4;          // per-call metadata slots (pinned host + device)
@@ -426,6 +433,13 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     if (!tma_api_init(&e->tma)) return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     WF_CUDA(e, gemm_bf16_configure());
     WF_CUDA(e, attention_bf16_configure());
+    // WF_GEMM_TAIL_SPLIT=1 lets residual GEMMs cut the tiles of their last, partial round along K
+    // (faster when M is small; the float32 additions then land in an order that varies from run
+    // to run, so results are no longer bit-reproducible).  Off unless asked for.
+    const char* pdl_env = getenv("WF_PDL");
+    pdl_set(!(pdl_env != nullptr && pdl_env[0] == '0'));
+    const char* split_env = getenv("WF_GEMM_TAIL_SPLIT");
+    gemm_bf16_set_tail_split(split_env != nullptr && split_env[0] == '1');
   }
   // tables
   WF_TRY(dev_alloc<float>(e, &e->dft_basis, 2L * kFold * kBasisCols));

@@ -132,6 +132,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();  // the set-up above overlapped the previous kernel's tail; qkv is read from here on
+  griddep_launch_dependents();
 
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
@@ -428,8 +430,8 @@ void launch_attention_bf16(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv
   const int n_head = d_model / kHeadDim;
   const int n_items = n_work * n_head;
   const int grid = n_items < num_sms ? n_items : num_sms;
-  attention_tc_kernel<<<grid, kAttnThreads, kAttnSmem, s>>>(tmap_q, tmap_kv, out, meta, ml, n_items, n_head, d_model,
-                                                            err_flag);
+  launch_dependent(attention_tc_kernel, dim3(grid), dim3(kAttnThreads), kAttnSmem, s, 1, tmap_q, tmap_kv, out, meta, ml,
+                   n_items, n_head, d_model, err_flag);
 }
 
 }  // namespace wf

@@ -12,6 +12,8 @@
 //               while the MMA warp already fills the other accumulator buffer.
 // Every mbarrier wait is bounded; on a timeout the CTA sets an error word, drains its own
 // TMA copies, frees its tensor memory and returns.
+#include <algorithm>
+
 #include "wf_internal.h"
 #include "wf_epilogue.cuh"
 #include "wf_ptx.cuh"
@@ -41,11 +43,11 @@ struct GemmCfg {
 // required: columns at or beyond N are computed from a clamped bias index and never stored).
 template <int EPI>
 __device__ __forceinline__ void bias_act32(const EpiParams& ep, int col0, int N, const uint32_t (&acc)[32],
-                                           float (&v)[32]) {
+                                           float (&v)[32], bool with_bias = true) {
 #pragma unroll
   for (int g = 0; g < 8; ++g) {
     int col = col0 + 4 * g;
-    float4 b = col < N ? __ldg(reinterpret_cast<const float4*>(ep.bias + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 b = (col < N && with_bias) ? __ldg(reinterpret_cast<const float4*>(ep.bias + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
     v[4 * g + 0] = __uint_as_float(acc[4 * g + 0]) + b.x;
     v[4 * g + 1] = __uint_as_float(acc[4 * g + 1]) + b.y;
     v[4 * g + 2] = __uint_as_float(acc[4 * g + 2]) + b.z;
@@ -80,7 +82,7 @@ __device__ __forceinline__ void conv2_store32(const EpiParams& ep, long row, lon
 template <int BN, int EPI>
 __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtensorMap* tmap_c, uint32_t t_row, int m0,
                                               int n0, long M, int N, int quarter, int lane, uint32_t stage_base,
-                                              uint32_t& piece) {
+                                              uint32_t& piece, bool with_bias = true) {
   const long row = (long)m0 + quarter * 32 + lane;
   if (EPI == kEpiConv2) {
 #pragma unroll 1
@@ -103,16 +105,17 @@ __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtenso
       float v[32];
       tmem_ld_32x32(t_row + c * 32, a32);
       tmem_ld_wait();
-      bias_act32<EPI>(ep, n0 + c * 32, N, a32, v);
+      bias_act32<EPI>(ep, n0 + c * 32, N, a32, v, with_bias);
 #pragma unroll
       for (int j = 0; j < 8; ++j)
         st_shared_v4(buf + lane * 128 + ((j ^ (lane & 7)) << 4), __float_as_uint(v[4 * j]),
                      __float_as_uint(v[4 * j + 1]), __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0 && n0 + c * 32 < N && (long)m0 + quarter * 32 < M) {
-        tma_reduce_add_2d(tmap_c, buf, n0 + c * 32, m0 + quarter * 32);
-        bulk_commit();
+      if (lane == 0) {
+        if (n0 + c * 32 < N && (long)m0 + quarter * 32 < M) tma_reduce_add_2d(tmap_c, buf, n0 + c * 32, m0 + quarter * 32);
+        bulk_commit();  // one group per piece, empty when the piece lies outside the matrix: wait_read<1>
+                        // above counts groups to know that the copy two pieces back has let go of its buffer
       }
       ++piece;
     }
@@ -149,9 +152,9 @@ __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtenso
       }
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0 && n0 + c * 64 < N && (long)m0 + quarter * 32 < M) {
-        tma_store_2d(tmap_c, buf, n0 + c * 64, m0 + quarter * 32);
-        bulk_commit();
+      if (lane == 0) {
+        if (n0 + c * 64 < N && (long)m0 + quarter * 32 < M) tma_store_2d(tmap_c, buf, n0 + c * 64, m0 + quarter * 32);
+        bulk_commit();  // one group per piece, also when nothing was stored (see above)
       }
       ++piece;
     }
@@ -198,6 +201,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();  // everything above overlapped the previous kernel's tail; its output is needed from here on
+  griddep_launch_dependents();
 
   const int num_m = (int)((M + kBM - 1) / kBM);
   const int num_n = (N + BN - 1) / BN;
@@ -303,6 +308,21 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
   }
 }
 
+// Work units of the CTA-pair kernel.  Tiles are dealt round-robin to the pairs; the tiles of the
+// last, partial round are cut along K into `split` parts (only for the residual epilogue, whose
+// float32 add-reduction makes partial sums free to combine), so that every pair has work in
+// that round too.  Unit u < full is the whole tile u; the others are (tile, K part) pairs, with
+// the bias added by part 0 alone.
+struct GemmUnit {
+  int tile, kb0, kb1;
+  bool first;
+};
+__device__ __forceinline__ GemmUnit gemm_unit(int u, int full, int rem, int split, int num_k) {
+  if (u < full) return GemmUnit{u, 0, num_k, true};
+  const int v = u - full, part = v / rem;
+  return GemmUnit{full + v % rem, part * num_k / split, (part + 1) * num_k / split, part == 0};
+}
+
 // ---------------------------------------------------------------------------------------------
 // The same GEMM on CTA pairs (thread-block clusters of two, tcgen05 cta_group::2): one MMA
 // covers a 256 x 256 tile, 128 rows per CTA, and each CTA stages only half of the W tile
@@ -314,7 +334,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
 template <int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
     const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-    const __grid_constant__ CUtensorMap tmap_c, long M, int N, int K, int a_cols, EpiParams ep, int* err_flag) {
+    const __grid_constant__ CUtensorMap tmap_c, long M, int N, int K, int a_cols, EpiParams ep, int* err_flag,
+    int tail_split) {
   constexpr int BN = 256;
   constexpr int kStages = 6;
   constexpr int kABytes = kBM * kBK * 2;          // this CTA's 128 rows of A
@@ -357,11 +378,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
   cluster_sync_all();  // barriers of both CTAs are initialised before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();  // everything above overlapped the previous kernel's tail; its output is needed from here on
+  griddep_launch_dependents();
 
   const int num_m = (int)((M + 2 * kBM - 1) / (2 * kBM));
   const int num_n = (N + BN - 1) / BN;
   const int num_k = (K + kBK - 1) / kBK;
   const int num_tiles = num_m * num_n;
+  const int full_tiles = (num_tiles / n_pairs) * n_pairs, rem_tiles = num_tiles - full_tiles;
+  const int num_units = full_tiles + rem_tiles * tail_split;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -370,10 +395,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = pair_id; ok && tile < num_tiles; tile += n_pairs) {
-        const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
-        const int n0 = (tile % num_n) * BN + (int)rank * (BN / 2);
-        for (int kb = 0; kb < num_k; ++kb) {
+      for (int u = pair_id; ok && u < num_units; u += n_pairs) {
+        const GemmUnit w = gemm_unit(u, full_tiles, rem_tiles, tail_split, num_k);
+        const int m0 = (w.tile / num_n) * (2 * kBM) + (int)rank * kBM;
+        const int n0 = (w.tile % num_n) * BN + (int)rank * (BN / 2);
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t leader_full = map_to_cta(full_bar(stage), 0);  // the leader CTA's barrier
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * kStageBytes);
@@ -394,11 +420,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int tile = pair_id; ok && tile < num_tiles; tile += n_pairs) {
+      for (int u = pair_id; ok && u < num_units; u += n_pairs) {
+        const GemmUnit w = gemm_unit(u, full_tiles, rem_tiles, tail_split, num_k);
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < num_k; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * kStageBytes;
@@ -406,7 +433,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
           const uint64_t bdesc = umma_desc_k_sw128(sa + kABytes);
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k)
-            umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > w.kb0 || k != 0) ? 1u : 0u);
           umma_commit_pair(empty_bar(stage), 3);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -422,9 +449,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
     uint32_t piece = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (int tile = pair_id; tile < num_tiles; tile += n_pairs) {
-      const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
-      const int n0 = (tile % num_n) * BN;
+    for (int u = pair_id; u < num_units; u += n_pairs) {
+      const GemmUnit w = gemm_unit(u, full_tiles, rem_tiles, tail_split, num_k);
+      const int m0 = (w.tile / num_n) * (2 * kBM) + (int)rank * kBM;
+      const int n0 = (w.tile % num_n) * BN;
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) {
@@ -433,7 +461,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
       }
       tc_fence_after();
       epilogue_tile<BN, EPI>(ep, &tmap_c, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN), m0, n0,
-                             M, N, quarter, lane, stage_base, piece);
+                             M, N, quarter, lane, stage_base, piece, w.first);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
@@ -524,34 +552,36 @@ static void launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUten
                        int a_cols, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
   const long tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
   const int grid = (int)(tiles < num_sms ? tiles : num_sms);
-  gemm_bf16_kernel<BN, EPI><<<grid, kGemmThreads, GemmCfg<BN>::kSmemBytes, s>>>(ta, tb, tc, M, N, K, a_cols, ep,
-                                                                                 err_flag);
+  launch_dependent(gemm_bf16_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::kSmemBytes, s, 1, ta, tb, tc,
+                   M, N, K, a_cols, ep, err_flag);
 }
+
+// pair = 1: CTA-pair kernel (W maps must then use 128-row boxes); 0: single-CTA kernel
+static int g_gemm_use_pair = 1;
+static int g_gemm_tail_split = 0;
+void gemm_bf16_set_pair(int on) { g_gemm_use_pair = on; }
+int gemm_bf16_uses_pair() { return g_gemm_use_pair; }
+void gemm_bf16_set_tail_split(int on) { g_gemm_tail_split = on; }
 
 template <int EPI>
 static void launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
                         int a_cols, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
   const long tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + 255) / 256);
-  const long pairs = tiles < num_sms / 2 ? tiles : num_sms / 2;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(2 * pairs));
-  cfg.blockDim = dim3(kGemmThreads);
-  cfg.dynamicSmemBytes = kPairSmemBytes;
-  cfg.stream = s;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = 2;
-  attr.val.clusterDim.y = 1;
-  attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  cudaLaunchKernelEx(&cfg, gemm_bf16_pair_kernel<EPI>, ta, tb, tc, M, N, K, a_cols, ep, err_flag);
+  const long max_pairs = num_sms / 2;
+  long pairs = tiles < max_pairs ? tiles : max_pairs;
+  // the residual epilogue lets the tiles of the last, partial round be cut along K (see GemmUnit);
+  // with fewer tiles than pairs that round is the only one, and more pairs are launched for it
+  int tail_split = 1;
+  if (EPI == kEpiBiasResid && g_gemm_tail_split) {
+    const long num_k = (K + kBK - 1) / kBK;
+    if (tiles < max_pairs) pairs = std::min(max_pairs, tiles * num_k);
+    const long rem = tiles % pairs;
+    if (rem > 0) tail_split = (int)std::max(1L, std::min(pairs / rem, num_k));
+    if (tiles < max_pairs) pairs = tiles * tail_split;
+  }
+  launch_dependent(gemm_bf16_pair_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(kGemmThreads), kPairSmemBytes, s, 2,
+                   ta, tb, tc, M, N, K, a_cols, ep, err_flag, tail_split);
 }
-
-// pair = 1: CTA-pair kernel (W maps must then use 128-row boxes); 0: single-CTA kernel
-static int g_gemm_use_pair = 1;
-void gemm_bf16_set_pair(int on) { g_gemm_use_pair = on; }
-int gemm_bf16_uses_pair() { return g_gemm_use_pair; }
 
 void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
                       int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {

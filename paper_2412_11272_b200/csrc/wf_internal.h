@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "../../include/wf_encoder.h"
 
 namespace wf {
@@ -48,6 +50,39 @@ struct MetaLayout {
   int attn_work;    // [n_attn_work] pairs (sequence, first query row within the sequence)
   int total;
 };
+
+// ---- kernel launch with optional cluster size and programmatic stream serialization.
+// With the latter the kernel may begin (set up barriers, allocate tensor memory) while the kernel
+// before it in the stream drains; it must call ptx::griddep_wait() before it touches global
+// memory.  pdl_enabled() is process-wide (wf_api.cu; on unless WF_PDL=0 in the environment).
+int pdl_enabled();
+void pdl_set(int on);
+template <typename... P, typename... A>
+inline cudaError_t launch_dependent(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    int cluster_x, A&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attrs[2];
+  unsigned n = 0;
+  if (cluster_x > 1) {
+    attrs[n].id = cudaLaunchAttributeClusterDimension;
+    attrs[n].val.clusterDim.x = (unsigned)cluster_x;
+    attrs[n].val.clusterDim.y = 1;
+    attrs[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (pdl_enabled()) {
+    attrs[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = attrs;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<A>(args)...);
+}
 
 // ---- tables (wf_frontend.cu)
 void launch_build_tables(float* dft_basis /*[2][kFold][kBasisCols]*/, float* pe, int n_ctx, int d,
@@ -95,6 +130,9 @@ cudaError_t gemm_bf16_configure();
 // 1 (default): CTA-pair kernel, W tensor maps need 128-row boxes; 0: single-CTA kernel, 256-row boxes
 int gemm_bf16_uses_pair();
 void gemm_bf16_set_pair(int on);
+// 1: residual-epilogue GEMMs cut the tiles of their last, partial round along K (default 0:
+// the order of the float32 residual additions, and with it every output bit, is then fixed)
+void gemm_bf16_set_tail_split(int on);
 // a_cols: stored row length of A in elements (K for a plain GEMM; smaller when one GEMM row
 // spans several consecutive stored rows, which must then be a multiple of 64).
 // tc: output map (bf16 out for kEpiBias/kEpiBiasGelu/kEpiConv1, float32 residual for

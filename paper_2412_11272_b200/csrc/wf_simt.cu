@@ -1,6 +1,7 @@
 // float32 SIMT kernels (the float32 encoder path), LayerNorm, and weight-layout conversion.
 #include "wf_internal.h"
 #include "wf_epilogue.cuh"
+#include "wf_ptx.cuh"
 
 namespace wf {
 
@@ -77,6 +78,8 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const float* __restrict_
                                                         const float* __restrict__ g,
                                                         const float* __restrict__ b,
                                                         OutT* __restrict__ out, long M) {
+  ptx::griddep_wait();
+  ptx::griddep_launch_dependents();
   const long row = (long)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= M) return;
@@ -120,16 +123,16 @@ static void layernorm_dispatch(const float* x, const float* g, const float* b, O
                                cudaStream_t s) {
   unsigned grid = (unsigned)((M + 7) / 8);
   switch (d / 128) {
-    case 1: layernorm_kernel<1, OutT><<<grid, 256, 0, s>>>(x, g, b, out, M); break;
-    case 2: layernorm_kernel<2, OutT><<<grid, 256, 0, s>>>(x, g, b, out, M); break;
-    case 3: layernorm_kernel<3, OutT><<<grid, 256, 0, s>>>(x, g, b, out, M); break;
-    case 4: layernorm_kernel<4, OutT><<<grid, 256, 0, s>>>(x, g, b, out, M); break;
-    case 5: layernorm_kernel<5, OutT><<<grid, 256, 0, s>>>(x, g, b, out, M); break;
-    case 6: layernorm_kernel<6, OutT><<<grid, 256, 0, s>>>(x, g, b, out, M); break;
-    case 7: layernorm_kernel<7, OutT><<<grid, 256, 0, s>>>(x, g, b, out, M); break;
-    case 8: layernorm_kernel<8, OutT><<<grid, 256, 0, s>>>(x, g, b, out, M); break;
-    case 9: layernorm_kernel<9, OutT><<<grid, 256, 0, s>>>(x, g, b, out, M); break;
-    case 10: layernorm_kernel<10, OutT><<<grid, 256, 0, s>>>(x, g, b, out, M); break;
+    case 1: launch_dependent(layernorm_kernel<1, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
+    case 2: launch_dependent(layernorm_kernel<2, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
+    case 3: launch_dependent(layernorm_kernel<3, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
+    case 4: launch_dependent(layernorm_kernel<4, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
+    case 5: launch_dependent(layernorm_kernel<5, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
+    case 6: launch_dependent(layernorm_kernel<6, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
+    case 7: launch_dependent(layernorm_kernel<7, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
+    case 8: launch_dependent(layernorm_kernel<8, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
+    case 9: launch_dependent(layernorm_kernel<9, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
+    case 10: launch_dependent(layernorm_kernel<10, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
     default: break;  // create() rejects d_model > 1280
   }
 }

@@ -194,6 +194,59 @@ def test_tcgen05_gemm_matches_fp64(M, N, K, mode):
     enc.close()
 
 
+@pytest.mark.parametrize("mode", [0, 2])
+def test_tcgen05_gemm_ragged_last_tile_repeated(mode):
+    """M leaves whole 32-row groups of the last tile outside the matrix and N leaves 32-column
+    pieces outside: the epilogue warps that own them store nothing there, and must still not
+    reuse a staging buffer that the previous tile's last copy is reading.  That is a race, so
+    the launch is repeated; every repetition is compared in full (on the device)."""
+    shape = _small("bf16", n_layer=0)
+    enc = make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000)
+    M, N, K = 20000, 1184, 640
+    rng = np.random.default_rng(5)
+    A = I.round_to_bf16(rng.normal(size=(M, K)).astype(np.float32))
+    Wm = I.round_to_bf16((rng.normal(size=(N, K)) / math.sqrt(K)).astype(np.float32))
+    bias = rng.normal(size=N).astype(np.float32)
+    resid = rng.normal(size=(M, N)).astype(np.float32)
+    ref = A.astype(np.float64) @ Wm.astype(np.float64).T + bias + (resid if mode == 2 else 0.0)
+    d_ref, d_resid = _dev(ref.astype(np.float32)), _dev(resid)
+    dA, dW, db = _dev(A, torch.bfloat16), _dev(Wm, torch.bfloat16), _dev(bias)
+    worst = 0.0
+    for _ in range(25):
+        if mode == 2:
+            C = d_resid.clone()
+            enc.wf_gemm_bf16(dA, dW, db, 2, C)
+        else:
+            C = enc.wf_gemm_bf16(dA, dW, db, 0)
+        err = (C.float() - d_ref).abs()
+        worst = max(worst, float((err / (d_ref.abs() + 1.0)).max()) if mode == 0 else float(err.max()))
+    enc.wf_check()
+    assert worst < (2.0 ** -8 if mode == 0 else 2e-5 * math.sqrt(K) + 1e-5), worst
+    enc.close()
+
+
+@pytest.mark.parametrize("M,N,K", [(4097, 1280, 1280), (300, 256, 5120), (20000, 1280, 640)])
+def test_tcgen05_gemm_tail_split_matches_fp64(M, N, K, monkeypatch):
+    """Residual GEMM with the K split of the last partial round of tiles switched on (85 tiles on
+    74 CTA pairs; fewer tiles than pairs; a split limited by the number of K blocks)."""
+    monkeypatch.setenv("WF_GEMM_TAIL_SPLIT", "1")
+    shape = _small("bf16", n_layer=0)
+    enc = make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000)
+    rng = np.random.default_rng(M + N + K)
+    A = I.round_to_bf16(rng.normal(size=(M, K)).astype(np.float32))
+    Wm = I.round_to_bf16((rng.normal(size=(N, K)) / math.sqrt(K)).astype(np.float32))
+    bias = rng.normal(size=N).astype(np.float32)
+    resid = rng.normal(size=(M, N)).astype(np.float32)
+    ref = A.astype(np.float64) @ Wm.astype(np.float64).T + bias + resid
+    C = _dev(resid)
+    enc.wf_gemm_bf16(_dev(A, torch.bfloat16), _dev(Wm, torch.bfloat16), _dev(bias), 2, C)
+    enc.wf_check()
+    assert np.max(np.abs(to_np(C) - ref)) < 2e-5 * math.sqrt(K) + 1e-5
+    enc.close()
+    monkeypatch.delenv("WF_GEMM_TAIL_SPLIT")
+    make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000).close()     # back to the default
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_cross_kv_projection_matches_oracle(dtype):
     """Encoder output -> cross-attention keys/values of every decoder layer (one GEMM)."""
@@ -316,7 +369,7 @@ def test_bf16_base_config_matches_oracle():
     assert cu[-1] == M
     for i, r in oracle_hidden(batch, shape, W, hush).items():
         _check_bf16(got[cu[i]:cu[i + 1]], r)
-    # host-buffer entry point gives the same result
+    # host-buffer entry point gives the same result, bit for bit
     a_host = torch.as_tensor(batch.audio).pin_memory()
     o_host = torch.empty((M, shape.d_model), dtype=torch.bfloat16).pin_memory()
     enc.wf_encode_host(a_host, batch.lengths, _dev(hush), o_host)
