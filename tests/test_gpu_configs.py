@@ -35,6 +35,12 @@ def _run(name, batch, hush_frames, picks, n_ctx=None):
     assert list(np.diff(cu)) == list(I.tokens_of(batch.lengths, hush_frames))
     got = to_np(out)
     assert np.isfinite(got).all()
+    # a property that holds at any size: the path has a fixed order of operations, so repeating the
+    # call reproduces every bit (a data race anywhere in the launch sequence shows up here)
+    first = out.clone()
+    for _ in range(3):
+        again, _ = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush) if hush_frames else None)
+        assert torch.equal(again, first), name
     refs = oracle_hidden(batch, shape, W, hush, only=set(picks))
     for i, ref in refs.items():
         g = got[cu[i]:cu[i + 1]]
