@@ -85,7 +85,7 @@ struct Plan {
   int B;
   long total_samples;
   int total_frames, total_prows, total_tokens;
-  int n_fe_tiles, n_work, max_prows_seq;
+  int n_fe_tiles, n_work, n_work_b, max_prows_seq;
   MetaLayout ml;
 };
 
@@ -165,6 +165,42 @@ class Prof {
   ProfEvent* ev_;
 };
 
+// Attention work list for sequences in `order` (tok[i] .. tok[i+1] are sequence i's tokens), as
+// (sequence, first query row) pairs written at `dst`.  float32 kernel: one entry per 16 rows.
+// bf16 kernel: first the entries of 256 consecutive rows whose two 128-row tiles are both
+// non-empty (*n_a of them), then one entry for the odd last tile of every sequence that has one
+// (*n_b; those run two heads side by side).
+void build_attn_work(const int* tok, const std::vector<int>& order, bool bf16, int* dst, int* n_a, int* n_b) {
+  int nw = 0;
+  *n_b = 0;
+  if (!bf16) {
+    for (int i : order)
+      for (int q0 = 0; q0 < tok[i + 1] - tok[i]; q0 += 16) {
+        dst[2 * nw] = i;
+        dst[2 * nw + 1] = q0;
+        ++nw;
+      }
+    *n_a = nw;
+    return;
+  }
+  for (int i : order)
+    for (int q0 = 0; q0 + 128 < tok[i + 1] - tok[i]; q0 += 256) {
+      dst[2 * nw] = i;
+      dst[2 * nw + 1] = q0;
+      ++nw;
+    }
+  *n_a = nw;
+  for (int i : order) {
+    const int tiles = (tok[i + 1] - tok[i] + 127) / 128;
+    if (tiles & 1) {
+      dst[2 * nw] = i;
+      dst[2 * nw + 1] = (tiles - 1) * 128;
+      ++nw;
+      ++*n_b;
+    }
+  }
+}
+
 // Builds prefix sums, the padded-row layout and the work lists for one call into `hm`
 // (host ints), validating every length.  `frames_given`: `len` holds frame counts, not samples.
 wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Plan* p, int* hm,
@@ -217,24 +253,15 @@ wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Pl
   hm[ml.prow_off + B] = (int)prows;
   hm[ml.tok_off + B] = (int)tokens;
   hm[ml.fe_tile_off + B] = (int)tiles;
-  // attention work list: (sequence, first query row), longest sequences first
-  const int qt = e->bf16 ? 256 : 16;
+  // attention work list, longest sequences first
   std::vector<int> order(B);
   for (int i = 0; i < B; ++i) order[i] = i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
     return hm[ml.tok_off + a + 1] - hm[ml.tok_off + a] > hm[ml.tok_off + b + 1] - hm[ml.tok_off + b];
   });
-  int nw = 0;
-  for (int oi = 0; build_work && oi < B; ++oi) {
-    int i = order[oi];
-    int n = hm[ml.tok_off + i + 1] - hm[ml.tok_off + i];
-    for (int q0 = 0; q0 < n; q0 += qt) {
-      hm[ml.attn_work + 2 * nw] = i;
-      hm[ml.attn_work + 2 * nw + 1] = q0;
-      ++nw;
-    }
-  }
-  ml.total = ml.attn_work + 2 * nw;
+  int nw = 0, nw_b = 0;
+  if (build_work) build_attn_work(hm + ml.tok_off, order, e->bf16, hm + ml.attn_work, &nw, &nw_b);
+  ml.total = ml.attn_work + 2 * (nw + nw_b);
   p->B = B;
   p->total_samples = samples;
   p->total_frames = (int)frames;
@@ -242,6 +269,7 @@ wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Pl
   p->total_tokens = (int)tokens;
   p->n_fe_tiles = (int)tiles;
   p->n_work = nw;
+  p->n_work_b = nw_b;
   p->max_prows_seq = max_pr;
   return WF_OK;
 }
@@ -311,7 +339,7 @@ wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidde
     }
     {
       Prof pr(e, 5, s);
-      if (e->bf16) launch_attention_bf16(e->tm_qkv, e->tm_qkv_kv, (__nv_bfloat16*)e->attn, meta, p.ml, p.n_work, d, e->err_flag, e->num_sms, s);
+      if (e->bf16) launch_attention_bf16(e->tm_qkv, e->tm_qkv_kv, (__nv_bfloat16*)e->attn, meta, p.ml, p.n_work, p.n_work_b, d, e->err_flag, e->num_sms, s);
       else launch_attention_f32((const float*)e->qkv, (float*)e->attn, meta, p.ml, p.n_work, d, s);
     }
     {
@@ -784,15 +812,11 @@ wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, in
   ml.tok_off = 0;
   ml.attn_work = B + 1;
   for (int i = 0; i <= B; ++i) hm[i] = cu_seqlens[i];
-  const int qt = e->bf16 ? 256 : 16;
-  int nw = 0;
-  for (int i = 0; i < B; ++i)
-    for (int q0 = 0; q0 < cu_seqlens[i + 1] - cu_seqlens[i]; q0 += qt) {
-      hm[ml.attn_work + 2 * nw] = i;
-      hm[ml.attn_work + 2 * nw + 1] = q0;
-      ++nw;
-    }
-  ml.total = ml.attn_work + 2 * nw;
+  std::vector<int> order(B);
+  for (int i = 0; i < B; ++i) order[i] = i;
+  int nw = 0, nw_b = 0;
+  build_attn_work(hm, order, e->bf16, hm + ml.attn_work, &nw, &nw_b);
+  ml.total = ml.attn_work + 2 * (nw + nw_b);
   Plan p{};
   p.ml = ml;
   st = ring_upload(e, slot, p, s);
@@ -804,7 +828,7 @@ wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, in
       if (!make_tmap_bf16(e->tma, &tq, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 128) ||
           !make_tmap_bf16(e->tma, &tkv, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 96))
         return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected the qkv tensor map");
-      launch_attention_bf16(tq, tkv, (__nv_bfloat16*)out, e->meta_dev[slot], ml, nw, e->cfg.d_model, e->err_flag, e->num_sms, s);
+      launch_attention_bf16(tq, tkv, (__nv_bfloat16*)out, e->meta_dev[slot], ml, nw, nw_b, e->cfg.d_model, e->err_flag, e->num_sms, s);
     }
     else launch_attention_f32((const float*)qkv, (float*)out, e->meta_dev[slot], ml, nw, e->cfg.d_model, s);
   }

@@ -1,7 +1,10 @@
 // Non-causal variable-length attention on the 5th-generation tensor cores (bf16, head dim 64).
 //
-// A persistent CTA (352 threads) walks a list of work items; one item = up to 256 query rows
-// (two tiles of 128) of one (sequence, head); keys are consumed 96 at a time.  Roles:
+// A persistent CTA (352 threads) walks a list of work items.  An item is two tiles of 128 query
+// rows that run side by side: either 256 consecutive rows of one (sequence, head), which share
+// every K / V stage, or -- for the odd last tile of a sequence -- the same 128 rows of two
+// neighbouring heads, each tile with K / V stages of its own.  Keys are consumed 96 at a time.
+// Roles:
 //   warps 0-3 / 4-7  softmax for query tile 0 / 1, one thread per query row.  A step loads the
 //                    96 scores of its row from tensor memory once, releases the score buffer,
 //                    takes the row maximum, exponentiates and writes the probabilities back to
@@ -12,14 +15,15 @@
 //                    maximum exceeds it by more than 2^8 -- the final O / l does not depend on
 //                    that choice.  In steady state the softmax never waits for the tensor pipe.
 //   warp 8           one lane issues the TMA loads: Q tiles once per item, K and V tiles of 96
-//                    keys through two 4-stage rings.
+//                    keys through two rings of kKvStages stages.
 //   warps 9, 10      MMA issue for query tile 0 / 1 (warp 9 also owns the tensor-memory
 //                    allocation).  The whole warp runs the loop so that descriptors stay in
 //                    uniform registers; one elected lane issues S = Q K^T (128x96x64, operands in
 //                    shared memory) as soon as the softmax has read the previous scores, and
 //                    O += P V (128x64x96, P from tensor memory, V from shared memory as an
 //                    MN-major operand) when the probabilities are in place.  A K / V stage is
-//                    released when both tiles' MMAs on it have completed (barriers count two).
+//                    released by two arrivals: one per tile when the tiles share it, both from
+//                    the one tile that uses it otherwise.
 // Keys are addressed through the token prefix sums: a key tile that runs past the end of its
 // sequence is masked in the softmax, so no padded token ever contributes.
 // Tensor-memory columns per query tile t (base 256 t): S [0,96) f32; P0 [96,144), P1 [144,192)
@@ -35,7 +39,7 @@ namespace {
 
 constexpr int kTQ = 128;          // query rows per tile
 constexpr int kTK = 96;           // keys per step
-constexpr int kKvStages = 4;
+constexpr int kKvStages = 6;
 constexpr int kQBytes = kTQ * 64 * 2;      // 16 KB
 constexpr int kKvBytes = kTK * 64 * 2;     // 12 KB
 constexpr int kAttnThreads = 352;
@@ -62,20 +66,36 @@ __device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr) {
 }
 
 struct Item {
-  int tok0, n, q0, head, n_kv;
-  bool two;
+  int tok0, n, q0, q1, head, head1, n_kv;  // tile 1 covers rows q1.. of head1
+  bool two;    // tile 1 has work
+  bool split;  // the tiles belong to different heads: K / V stages alternate between them
 };
 
-__device__ __forceinline__ Item load_item(const int* __restrict__ meta, const MetaLayout& ml, int it, int n_head) {
+// Items [0, n_work_a * n_head): work entry = 256 consecutive rows (both tiles non-empty), one item
+// per head.  The rest: work entry = the odd last tile of a sequence, one item per pair of heads
+// (a last unpaired head runs as a single tile).
+__device__ __forceinline__ Item load_item(const int* __restrict__ meta, const MetaLayout& ml, int it, int n_head,
+                                          int n_work_a) {
   Item w;
-  const int work = it / n_head;
-  w.head = it - work * n_head;
+  int work;
+  if (it < n_work_a * n_head) {
+    work = it / n_head;
+    w.head = w.head1 = it - work * n_head;
+    w.two = true;
+    w.split = false;
+  } else {
+    const int itb = it - n_work_a * n_head, hp = (n_head + 1) >> 1;
+    work = n_work_a + itb / hp;
+    w.head = 2 * (itb % hp);
+    w.two = w.split = w.head + 1 < n_head;
+    w.head1 = w.two ? w.head + 1 : w.head;
+  }
   const int seq = meta[ml.attn_work + 2 * work];
   w.q0 = meta[ml.attn_work + 2 * work + 1];
+  w.q1 = w.split ? w.q0 : w.q0 + kTQ;
   w.tok0 = meta[ml.tok_off + seq];
   w.n = meta[ml.tok_off + seq + 1] - w.tok0;
   w.n_kv = (w.n + kTK - 1) / kTK;
-  w.two = w.q0 + kTQ < w.n;
   return w;
 }
 
@@ -83,8 +103,8 @@ __device__ __forceinline__ Item load_item(const int* __restrict__ meta, const Me
 
 __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
     const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
-    __nv_bfloat16* __restrict__ out, const int* __restrict__ meta, MetaLayout ml, int n_items, int n_head,
-    int d_model, int* err_flag) {
+    __nv_bfloat16* __restrict__ out, const int* __restrict__ meta, MetaLayout ml, int n_items, int n_work_a,
+    int n_head, int d_model, int* err_flag) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
@@ -143,23 +163,31 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
       uint32_t kc = 0, vc = 0, items = 0;
       bool ok = true;
       for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-        const Item w = load_item(meta, ml, it, n_head);
+        const Item w = load_item(meta, ml, it, n_head, n_work_a);
         if (!mbar_wait(q_free, (items & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         mbar_arrive_expect_tx(q_full, w.two ? 2 * kQBytes : kQBytes);
         tma_load_2d(sbase + kOffQ, &tmap_q, w.head * kHeadDim, w.tok0 + w.q0, q_full);
-        if (w.two) tma_load_2d(sbase + kOffQ + kQBytes, &tmap_q, w.head * kHeadDim, w.tok0 + w.q0 + kTQ, q_full);
-        for (int j = 0; j < w.n_kv; ++j) {
-          int s = kc % kKvStages;
-          if (!mbar_wait(k_free(s), ((kc / kKvStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          mbar_arrive_expect_tx(k_full(s), kKvBytes);
-          tma_load_2d(sbase + kOffK + s * kKvBytes, &tmap_kv, d_model + w.head * kHeadDim, w.tok0 + j * kTK, k_full(s));
-          ++kc;
-          s = vc % kKvStages;
-          if (!mbar_wait(v_free(s), ((vc / kKvStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          mbar_arrive_expect_tx(v_full(s), kKvBytes);
-          tma_load_2d(sbase + kOffV + s * kKvBytes, &tmap_kv, 2 * d_model + w.head * kHeadDim, w.tok0 + j * kTK, v_full(s));
-          ++vc;
+        if (w.two) tma_load_2d(sbase + kOffQ + kQBytes, &tmap_q, w.head1 * kHeadDim, w.tok0 + w.q1, q_full);
+        const int n_h = w.split ? 2 : 1;  // K / V stages per key step
+        for (int j = 0; ok && j < w.n_kv; ++j) {
+          for (int h = 0; h < n_h; ++h) {
+            const int s = kc % kKvStages;
+            if (!mbar_wait(k_free(s), ((kc / kKvStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+            mbar_arrive_expect_tx(k_full(s), kKvBytes);
+            tma_load_2d(sbase + kOffK + s * kKvBytes, &tmap_kv, d_model + (h ? w.head1 : w.head) * kHeadDim,
+                        w.tok0 + j * kTK, k_full(s));
+            ++kc;
+          }
+          for (int h = 0; ok && h < n_h; ++h) {
+            const int s = vc % kKvStages;
+            if (!mbar_wait(v_free(s), ((vc / kKvStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+            mbar_arrive_expect_tx(v_full(s), kKvBytes);
+            tma_load_2d(sbase + kOffV + s * kKvBytes, &tmap_kv, 2 * d_model + (h ? w.head1 : w.head) * kHeadDim,
+                        w.tok0 + j * kTK, v_full(s));
+            ++vc;
+          }
         }
+        if (!ok) break;
         ++items;
       }
       if (!ok) {
@@ -200,7 +228,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
       __syncwarp();
     };
     for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-      const Item w = load_item(meta, ml, it, n_head);
+      const Item w = load_item(meta, ml, it, n_head, n_work_a);
       if (t == 1 && !w.two) {
         // nothing to compute for this tile: release the stages in step with the other tile
         for (int j = 0; ok && j < w.n_kv; ++j) {
@@ -220,24 +248,33 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
         continue;
       }
       if (!wait_all(q_full, items & 1u)) { ok = false; break; }
-      int ks = kc % kKvStages;
-      if (!wait_all(k_full(ks), (kc / kKvStages) & 1u)) { ok = false; break; }
+      // with split tiles the stages alternate: this tile's are the t-th of every pair, and it alone
+      // gives both arrivals that release them
+      const uint32_t own = w.split ? (uint32_t)t : 0u, adv = w.split ? 2u : 1u;
+      auto release = [&](uint32_t bar) {
+        if (leader) {
+          umma_commit(bar);
+          if (w.split) umma_commit(bar);
+        }
+      };
+      int ks = (kc + own) % kKvStages;
+      if (!wait_all(k_full(ks), ((kc + own) / kKvStages) & 1u)) { ok = false; break; }
       tc_fence_after();
       issue_s(ks);  // the score buffer is free: its last reader arrived on s_free (waited below)
-      if (leader) umma_commit(k_free(ks));
-      ++kc;
+      release(k_free(ks));
+      kc += adv;
       for (int j = 0; j < w.n_kv; ++j) {
         if (!wait_all(s_free(t), g & 1u)) { ok = false; break; }
         if (j + 1 < w.n_kv) {
-          ks = kc % kKvStages;
-          if (!wait_all(k_full(ks), (kc / kKvStages) & 1u)) { ok = false; break; }
+          ks = (kc + own) % kKvStages;
+          if (!wait_all(k_full(ks), ((kc + own) / kKvStages) & 1u)) { ok = false; break; }
           tc_fence_after();
           issue_s(ks);
-          if (leader) umma_commit(k_free(ks));
-          ++kc;
+          release(k_free(ks));
+          kc += adv;
         }
-        const int vs = vc % kKvStages;
-        if (!wait_all(v_full(vs), (vc / kKvStages) & 1u)) { ok = false; break; }
+        const int vs = (vc + own) % kKvStages;
+        if (!wait_all(v_full(vs), ((vc + own) / kKvStages) & 1u)) { ok = false; break; }
         const int k_steps = (min(kTK, w.n - j * kTK) + 15) >> 4;
         const uint32_t b = g & 1u;
         if (!wait_all(p_full(t, b), (g >> 1) & 1u)) { ok = false; break; }
@@ -254,10 +291,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
           if (k_steps > 4) umma_bf16_ts(tm_o, tm_p + 32, vd + 512, idesc_o, 1u);
           if (k_steps > 5) umma_bf16_ts(tm_o, tm_p + 40, vd + 640, idesc_o, 1u);
           umma_commit(o_full(t, b));
-          umma_commit(v_free(vs));
         }
+        release(v_free(vs));
         __syncwarp();
-        ++vc;
+        vc += adv;
         ++g;
       }
       if (!ok) break;
@@ -282,10 +319,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
     };
 
     for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-      const Item w = load_item(meta, ml, it, n_head);
+      const Item w = load_item(meta, ml, it, n_head, n_work_a);
       if (t == 1 && !w.two) continue;
       // a warp whose 32 rows all lie beyond the sequence keeps pace with the barriers only
-      const bool active = w.q0 + t * kTQ + (warp & 3) * 32 < w.n;
+      const int row0 = t ? w.q1 : w.q0;  // first query row of this tile
+      const bool active = row0 + (warp & 3) * 32 < w.n;
       float m_ref = -INFINITY, l_run = 0.f;
 
       for (int j = 0; j < w.n_kv; ++j) {
@@ -379,10 +417,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
       }
       if (!wait_warp(o_full(t, (g - 1) & 1u), ((g - 1) >> 1) & 1u)) { ok = false; break; }
       tc_fence_after();
-      const int q = w.q0 + t * kTQ + r;
+      const int q = row0 + r;
       if (active) {
         const float inv = 1.0f / l_run;
-        __nv_bfloat16* dst = out + (long)(w.tok0 + q) * d_model + w.head * kHeadDim;
+        __nv_bfloat16* dst = out + (long)(w.tok0 + q) * d_model + (t ? w.head1 : w.head) * kHeadDim;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t a[16];
@@ -424,14 +462,14 @@ cudaError_t attention_bf16_configure() {
 }
 
 void launch_attention_bf16(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, __nv_bfloat16* out,
-                           const int* meta, MetaLayout ml, int n_work, int d_model, int* err_flag, int num_sms,
-                           cudaStream_t s) {
-  if (n_work <= 0) return;
+                           const int* meta, MetaLayout ml, int n_work_a, int n_work_b, int d_model, int* err_flag,
+                           int num_sms, cudaStream_t s) {
   const int n_head = d_model / kHeadDim;
-  const int n_items = n_work * n_head;
+  const int n_items = n_work_a * n_head + n_work_b * ((n_head + 1) / 2);
+  if (n_items <= 0) return;
   const int grid = n_items < num_sms ? n_items : num_sms;
   launch_dependent(attention_tc_kernel, dim3(grid), dim3(kAttnThreads), kAttnSmem, s, 1, tmap_q, tmap_kv, out, meta, ml,
-                   n_items, n_head, d_model, err_flag);
+                   n_items, n_work_a, n_head, d_model, err_flag);
 }
 
 }  // namespace wf
