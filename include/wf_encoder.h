@@ -165,6 +165,35 @@ wf_status wf_gemm_bf16(wf_encoder *enc, const void *A, const void *W, const floa
 wf_status wf_attention(wf_encoder *enc, const void *qkv, const int *cu_seqlens, int B, void *out,
                        void *stream);
 
+/* Resident stream windows (Sec. 3.2: every round a stream's audio buffer is extended at its end
+ * by the newly arrived audio and now and then cut at its front once a transcript segment is
+ * confirmed; Sec. 4.3.2: the buffer is re-encoded every round).  The library keeps each stream's
+ * window (samples and un-normalised log-mel rows) on the device, so that a round frames only the
+ * audio that is new: wf_streams_push recomputes just the frames whose 400 samples changed (the
+ * new ones, the two at the old end whose reflected tail became real audio and, after a cut, the
+ * first two), and wf_encode_streams runs the max / clamp / scale over the cached rows, appends the
+ * hush segment and encodes.  Results are identical, bit for bit, to wf_encode on the same windows.
+ *
+ * wf_streams_create: windows for n_streams streams of up to max_window_samples samples each
+ *   (rounded up to a multiple of 160); all windows start empty.  Device memory is allocated
+ *   here and released by wf_streams_destroy (which synchronises the device first).
+ * wf_streams_push: for each listed stream (ids host, B distinct ids), drop trim[i] samples at the
+ *   front (a multiple of 160, at most the window; trim may be NULL), then append n_new[i]
+ *   samples taken back to back from new_audio (dev float32).  The window must end up with at
+ *   least 401 samples (WF_ERR_TOO_SHORT) and at most its capacity (WF_ERR_CAPACITY); on an
+ *   error nothing is changed.
+ * wf_streams_length: samples currently in a stream's window (host bookkeeping, no sync).
+ * wf_encode_streams: as wf_encode, on the current windows of the listed streams, in the order
+ *   listed. */
+typedef struct wf_streams wf_streams;
+wf_status wf_streams_create(wf_encoder *enc, int n_streams, long max_window_samples, wf_streams **out);
+wf_status wf_streams_destroy(wf_streams *st);
+wf_status wf_streams_length(const wf_streams *st, int stream_id, long *samples);
+wf_status wf_streams_push(wf_streams *st, const int *ids, int B, const float *new_audio,
+                          const long *n_new, const long *trim, void *stream);
+wf_status wf_encode_streams(wf_streams *st, const int *ids, int B, const float *hush_mel,
+                            void *hidden_out, int *cu_seqlens_out, void *stream);
+
 /* wf_cross_kv: the cross-attention key and value projections of the encoder's output for every
  * decoder layer in one GEMM, kv = hidden W_kv^T + b_kv: the first thing prompt prefill (Sec. 3.2
  * "Operations", Sec. 4.3.2) needs from the encoding stage, and the same for every later decoding

@@ -54,7 +54,8 @@ _PER_LAYER = ("ln1_g", "ln1_b", "wq", "bq", "wk", "wv", "bv", "wo", "bo", "ln2_g
 
 EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_raw_hush", "wf_encode_mel", "wf_encode_host", "wf_check",
            "wf_encoder_destroy", "wf_last_error", "wf_profile_enable", "wf_profile_read",
-           "wf_gemm_bf16", "wf_attention", "wf_cross_kv", "wf_dtw", "wf_attention_f32_static",
+           "wf_gemm_bf16", "wf_attention", "wf_cross_kv", "wf_dtw",
+           "wf_streams_create", "wf_streams_destroy", "wf_streams_length", "wf_streams_push", "wf_encode_streams", "wf_attention_f32_static",
            "wf_beam_pruner_create", "wf_beam_pruner_step", "wf_beam_pruner_state", "wf_beam_pruner_destroy")
 
 _lib = None
@@ -84,6 +85,11 @@ def load_library() -> C.CDLL:
     lib.wf_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, C.c_long, C.c_int, C.c_int, C.c_int, vp]
     lib.wf_attention.argtypes = [vp, vp, ip, C.c_int, vp, vp]
     lib.wf_cross_kv.argtypes = [vp, vp, vp, vp, C.c_long, C.c_int, vp, vp]
+    lib.wf_streams_create.argtypes = [vp, C.c_int, C.c_long, C.POINTER(vp)]
+    lib.wf_streams_destroy.argtypes = [vp]
+    lib.wf_streams_length.argtypes = [vp, C.c_int, lp]
+    lib.wf_streams_push.argtypes = [vp, ip, C.c_int, vp, lp, lp, vp]
+    lib.wf_encode_streams.argtypes = [vp, ip, C.c_int, vp, vp, ip, vp]
     lib.wf_dtw.argtypes = [vp, vp, ip, ip, C.c_int, vp, vp, vp, vp]
     lib.wf_attention_f32_static.argtypes = [vp, ip, C.c_int, C.c_int, vp, vp]
     lib.wf_beam_pruner_create.argtypes = [ip, C.c_int, C.POINTER(C.c_ubyte), C.c_int, C.c_int, C.POINTER(vp)]
@@ -308,6 +314,59 @@ def wf_attention_f32_static(qkv: torch.Tensor, cu_seqlens, d_model: int, out: to
     if st != 0:
         raise WfError(st, "wf_attention_f32_static rejected its arguments or a CUDA call failed")
     return out
+
+
+class Streams:
+    """Resident windows of ``n_streams`` audio streams on an encoder's device (``wf_streams_*``)."""
+
+    def __init__(self, enc: Encoder, n_streams: int, max_window_samples: int):
+        self.enc = enc
+        self.handle = C.c_void_p()
+        enc._check(enc.lib.wf_streams_create(enc.handle, n_streams, max_window_samples, C.byref(self.handle)))
+
+    def close(self):
+        if self.handle:
+            self.enc.lib.wf_streams_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def wf_streams_length(self, stream_id: int) -> int:
+        n = C.c_long()
+        self.enc._check(self.enc.lib.wf_streams_length(self.handle, stream_id, C.byref(n)))
+        return n.value
+
+    def wf_streams_push(self, ids, new_audio: torch.Tensor | None, n_new, trim=None, stream=None):
+        """Drops ``trim[i]`` samples at the front of stream ``ids[i]`` and appends ``n_new[i]`` samples
+        taken back to back from ``new_audio`` (float32 CUDA)."""
+        idv = np.ascontiguousarray(np.asarray(ids, dtype=np.int32))
+        nn, nn_ptr = _longs(n_new)
+        tr_ptr = None
+        if trim is not None:
+            tr, tr_ptr = _longs(trim)
+        self.enc._check(self.enc.lib.wf_streams_push(
+            self.handle, idv.ctypes.data_as(C.POINTER(C.c_int)), len(idv),
+            new_audio.data_ptr() if new_audio is not None and new_audio.numel() else None, nn_ptr, tr_ptr,
+            _stream_ptr(stream)))
+
+    def wf_encode_streams(self, ids, hush_mel: torch.Tensor | None, out=None, stream=None):
+        """Encodes the current windows of the listed streams; returns (hidden, cu_seqlens)."""
+        enc = self.enc
+        idv = np.ascontiguousarray(np.asarray(ids, dtype=np.int32))
+        B = len(idv)
+        frames = np.array([self.wf_streams_length(int(i)) // 160 for i in idv], dtype=np.int64)
+        M = int(enc._tokens(frames).sum()) if B else 0
+        if out is None:
+            out = torch.empty((M, enc.d_model), dtype=enc.out_dtype, device=enc.device)
+        cu = np.zeros(B + 1, dtype=np.int32)
+        enc._check(enc.lib.wf_encode_streams(self.handle, idv.ctypes.data_as(C.POINTER(C.c_int)), B,
+                                             hush_mel.data_ptr() if hush_mel is not None else None, out.data_ptr(),
+                                             cu.ctypes.data_as(C.POINTER(C.c_int)), _stream_ptr(stream)))
+        return out, cu
 
 
 class BeamPruner:

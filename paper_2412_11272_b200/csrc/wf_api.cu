@@ -79,6 +79,19 @@ struct wf_encoder {
   size_t prof_used;
 };
 
+// Resident windows of `n` streams: samples and un-normalised log-mel rows on the device, lengths
+// on the host.
+struct wf_streams {
+  wf_encoder* enc;
+  int n;
+  long cap_samples;  // per stream, a multiple of the hop
+  long cap_frames;   // cap_samples / hop
+  float* audio;      // [n][cap_samples]
+  float* logmel;     // [n][cap_frames][n_mel]  log10 mel power, before the max / clamp / scale
+  int* scratch_max;  // [max_batch] sink for the front end's running maxima during a push
+  std::vector<long> len;
+};
+
 namespace {
 
 struct Plan {
@@ -217,6 +230,8 @@ wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Pl
   ml.tok_off = off; off += B + 1;
   ml.fe_tile_off = off; off += B + 1;
   ml.attn_work = off;
+  ml.fe_len = 0;
+  ml.fe_tiles = 0;
   long samples = 0, frames = 0, prows = 0, tokens = 0, tiles = 0;
   int max_pr = 0;
   for (int i = 0; i < B; ++i) {
@@ -726,6 +741,200 @@ wf_status wf_gemm_bf16(wf_encoder* e, const void* A, const void* W, const float*
   launch_gemm_bf16(ta, tb, tc, M, N, K, K, mode, ep, e->err_flag, e->num_sms, (cudaStream_t)stream);
   WF_CUDA(e, cudaGetLastError());
   return WF_OK;
+}
+
+wf_status wf_streams_create(wf_encoder* e, int n_streams, long max_window_samples, wf_streams** out) {
+  if (!e || !out) return WF_ERR_INVALID_ARG;
+  *out = nullptr;
+  const long cap = (max_window_samples + kHop - 1) / kHop * kHop;
+  if (n_streams < 1 || max_window_samples < kMinSamples || (double)n_streams * (double)cap * e->cfg.n_mel / kHop >= 2147483647.0 ||
+      (double)n_streams * (double)cap >= 2147483647.0)
+    return fail(e, WF_ERR_INVALID_ARG, "wf_streams_create: bad stream count or window size");
+  wf_streams* st = new (std::nothrow) wf_streams();
+  if (!st) return fail(e, WF_ERR_CUDA, "out of host memory");
+  st->enc = e;
+  st->n = n_streams;
+  st->cap_samples = cap;
+  st->cap_frames = cap / kHop;
+  st->audio = nullptr;
+  st->logmel = nullptr;
+  st->scratch_max = nullptr;
+  st->len.assign(n_streams, 0);
+  if (cudaMalloc(&st->audio, (size_t)n_streams * cap * sizeof(float)) != cudaSuccess ||
+      cudaMalloc(&st->logmel, (size_t)n_streams * st->cap_frames * e->cfg.n_mel * sizeof(float)) != cudaSuccess ||
+      cudaMalloc(&st->scratch_max, (size_t)e->cfg.max_batch * sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(st->audio);
+    cudaFree(st->logmel);
+    cudaFree(st->scratch_max);
+    delete st;
+    return fail(e, WF_ERR_CUDA, "wf_streams_create: out of device memory");
+  }
+  *out = st;
+  return WF_OK;
+}
+
+wf_status wf_streams_destroy(wf_streams* st) {
+  if (!st) return WF_OK;
+  cudaDeviceSynchronize();
+  cudaFree(st->audio);
+  cudaFree(st->logmel);
+  cudaFree(st->scratch_max);
+  delete st;
+  return WF_OK;
+}
+
+wf_status wf_streams_length(const wf_streams* st, int stream_id, long* samples) {
+  if (!st || !samples || stream_id < 0 || stream_id >= st->n) return WF_ERR_INVALID_ARG;
+  *samples = st->len[stream_id];
+  return WF_OK;
+}
+
+wf_status wf_streams_push(wf_streams* st, const int* ids, int B, const float* new_audio, const long* n_new,
+                          const long* trim, void* stream) {
+  if (!st) return WF_ERR_INVALID_ARG;
+  wf_encoder* e = st->enc;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (B < 0 || (B > 0 && (!ids || !n_new))) return fail(e, WF_ERR_INVALID_ARG, "wf_streams_push: NULL argument");
+  if (B > e->cfg.max_batch) return fail(e, WF_ERR_CAPACITY, "batch %d exceeds max_batch %d", B, e->cfg.max_batch);
+  if (B == 0) return WF_OK;
+  // validate everything before any state changes
+  std::vector<char> seen(st->n, 0);
+  long total_new = 0, max_new = 0;
+  int n_shift = 0, n_tiles = 0;
+  for (int i = 0; i < B; ++i) {
+    const int id = ids[i];
+    if (id < 0 || id >= st->n || seen[id]) return fail(e, WF_ERR_INVALID_ARG, "wf_streams_push: stream id %d out of range or repeated", id);
+    seen[id] = 1;
+    const long cut = trim ? trim[i] : 0, add = n_new[i], len = st->len[id];
+    if (cut < 0 || cut % kHop != 0 || cut > len || add < 0)
+      return fail(e, WF_ERR_INVALID_ARG, "wf_streams_push: stream %d: trim %ld (window %ld) or new sample count %ld", id, cut, len, add);
+    if (add > 0 && !new_audio) return fail(e, WF_ERR_INVALID_ARG, "wf_streams_push: new_audio is NULL");
+    const long nl = len - cut + add;
+    if (nl > st->cap_samples) return fail(e, WF_ERR_CAPACITY, "stream %d would hold %ld samples (capacity %ld)", id, nl, st->cap_samples);
+    if (nl < kMinSamples) return fail(e, WF_ERR_TOO_SHORT, "stream %d would hold %ld samples (need >= %d)", id, nl, kMinSamples);
+    total_new += add;
+    max_new = std::max(max_new, add);
+    if (cut > 0 && cut < len) ++n_shift;
+    // frames to compute: the two at the old end (their reflected tail is now real audio) and all
+    // new ones; after a cut also the first two (their reflected head changed)
+    const long T_new = nl / kHop, kept = (len - cut) / kHop;
+    const long from = std::max(0L, kept - 2);
+    if (cut > 0 && from > 0) ++n_tiles;
+    n_tiles += (int)((T_new - from + kFeFrames - 1) / kFeFrames);
+  }
+  const int need = 4 * (B + 1) + 2 * n_tiles + 6 * n_shift + 3 * B + 8;
+  if (need > e->meta_cap) return fail(e, WF_ERR_CAPACITY, "wf_streams_push: metadata capacity exceeded");
+  int slot;
+  wf_status rc = ring_acquire(e, &slot);
+  if (rc != WF_OK) return rc;
+  int* hm = e->meta_host[slot];
+  MetaLayout ml{};
+  ml.sample_off = 0;
+  ml.frames = B + 1;
+  ml.frame_off = 2 * (B + 1);
+  ml.fe_len = 3 * (B + 1);
+  ml.fe_tiles = 4 * (B + 1);
+  const int off_shift_a = ml.fe_tiles + 2 * n_tiles, off_shift_m = off_shift_a + 3 * n_shift;
+  const int off_append = off_shift_m + 3 * n_shift;
+  ml.total = off_append + 3 * B;
+  int it = 0, is = 0;
+  long src = 0;
+  const int n_mel = e->cfg.n_mel;
+  for (int i = 0; i < B; ++i) {
+    const int id = ids[i];
+    const long cut = trim ? trim[i] : 0, add = n_new[i], len = st->len[id];
+    const long nl = len - cut + add, T_new = nl / kHop, kept = (len - cut) / kHop;
+    hm[ml.sample_off + i] = (int)(id * st->cap_samples);
+    hm[ml.frames + i] = (int)T_new;
+    hm[ml.frame_off + i] = (int)(id * st->cap_frames);
+    hm[ml.fe_len + i] = (int)nl;
+    if (cut > 0 && cut < len) {
+      hm[off_shift_a + 3 * is] = (int)(id * st->cap_samples);
+      hm[off_shift_a + 3 * is + 1] = (int)cut;
+      hm[off_shift_a + 3 * is + 2] = (int)len;
+      hm[off_shift_m + 3 * is] = (int)(id * st->cap_frames * n_mel);
+      hm[off_shift_m + 3 * is + 1] = (int)(cut / kHop * n_mel);
+      hm[off_shift_m + 3 * is + 2] = (int)(len / kHop * n_mel);
+      ++is;
+    }
+    hm[off_append + 3 * i] = (int)(id * st->cap_samples + len - cut);
+    hm[off_append + 3 * i + 1] = (int)src;
+    hm[off_append + 3 * i + 2] = (int)add;
+    src += add;
+    const long from = std::max(0L, kept - 2);
+    if (cut > 0 && from > 0) {
+      hm[ml.fe_tiles + 2 * it] = i;
+      hm[ml.fe_tiles + 2 * it + 1] = 0;  // recomputes frames 0..63: the first two are the ones that changed
+      ++it;
+    }
+    for (long t0 = from; t0 < T_new; t0 += kFeFrames) {
+      hm[ml.fe_tiles + 2 * it] = i;
+      hm[ml.fe_tiles + 2 * it + 1] = (int)t0;
+      ++it;
+    }
+  }
+  hm[ml.sample_off + B] = hm[ml.frames + B] = hm[ml.frame_off + B] = 0;
+  Plan p{};
+  p.ml = ml;
+  rc = ring_upload(e, slot, p, s);
+  if (rc != WF_OK) return rc;
+  const int* meta = e->meta_dev[slot];
+  {
+    Prof pr(e, 0, s);
+    launch_stream_shift(st->audio, st->logmel, meta + off_shift_a, meta + off_shift_m, n_shift, s);
+    launch_stream_append(st->audio, new_audio, meta + off_append, B, (int)max_new, s);
+    launch_frontend(st->audio, meta, ml, B, it, e->dft_basis, e->mel_fb_t, n_mel, st->logmel, st->scratch_max, nullptr, 0, s);
+  }
+  WF_CUDA(e, cudaGetLastError());
+  for (int i = 0; i < B; ++i) st->len[ids[i]] += n_new[i] - (trim ? trim[i] : 0);
+  return ring_release(e, slot, s);
+}
+
+wf_status wf_encode_streams(wf_streams* st, const int* ids, int B, const float* hush, void* hidden_out,
+                            int* cu_out, void* stream) {
+  if (!st) return WF_ERR_INVALID_ARG;
+  wf_encoder* e = st->enc;
+  const wf_config& c = e->cfg;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (c.hush_frames > 0 && !hush) return fail(e, WF_ERR_INVALID_ARG, "hush_mel is NULL but hush_frames > 0");
+  if (B < 0 || (B > 0 && (!ids || !hidden_out))) return fail(e, WF_ERR_INVALID_ARG, "NULL input or output");
+  if (B > c.max_batch) return fail(e, WF_ERR_CAPACITY, "batch %d exceeds max_batch %d", B, c.max_batch);
+  std::vector<long> frames(std::max(B, 1));
+  for (int i = 0; i < B; ++i) {
+    if (ids[i] < 0 || ids[i] >= st->n) return fail(e, WF_ERR_INVALID_ARG, "stream id %d out of range", ids[i]);
+    if (st->len[ids[i]] < kMinSamples) return fail(e, WF_ERR_TOO_SHORT, "stream %d holds %ld samples", ids[i], st->len[ids[i]]);
+    frames[i] = st->len[ids[i]] / kHop;
+  }
+  int slot;
+  wf_status rc = ring_acquire(e, &slot);
+  if (rc != WF_OK) return rc;
+  Plan p;
+  rc = make_plan(e, frames.data(), true, B, &p, e->meta_host[slot]);
+  if (rc != WF_OK) return rc;
+  int* hm = e->meta_host[slot];
+  if (cu_out)
+    for (int i = 0; i <= B; ++i) cu_out[i] = hm[p.ml.tok_off + i];
+  if (B == 0) return WF_OK;
+  int max_T = 0;
+  for (int i = 0; i < B; ++i) {
+    hm[p.ml.frame_off + i] = (int)(ids[i] * st->cap_frames);  // rows are read from the resident windows
+    max_T = std::max(max_T, (int)frames[i]);
+  }
+  rc = ring_upload(e, slot, p, s);
+  if (rc != WF_OK) return rc;
+  const int* meta = e->meta_dev[slot];
+  void* zp = (uint8_t*)e->zp_alloc + (size_t)e->mel_ld * e->esz;
+  {
+    Prof pr(e, 1, s);
+    launch_fill_seq_max(e->seq_max, B, s);
+    launch_stream_max(st->logmel, meta, p.ml, B, max_T, c.n_mel, e->seq_max, s);
+    launch_normalise(st->logmel, e->seq_max, nullptr, meta, p.ml, B, p.max_prows_seq, c.n_mel, e->mel_ld,
+                     c.hush_frames, hush, zp, e->bf16 ? 1 : 0, 1, s);
+  }
+  rc = run_encoder(e, p, meta, hidden_out, s);
+  if (rc != WF_OK) return rc;
+  return ring_release(e, slot, s);
 }
 
 wf_status wf_cross_kv(wf_encoder* e, const void* hidden, const void* W_kv, const float* b_kv, long M,

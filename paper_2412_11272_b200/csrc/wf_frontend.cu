@@ -80,18 +80,24 @@ __global__ void __launch_bounds__(256) frontend_kernel(
   float* o_s = smem + kFeFrames * kFold;   // [64][200]
   float* p_s = smem;                       // [64][204] after the DFT
 
-  const int* tile_off = meta + ml.fe_tile_off;
-  int tile = blockIdx.x;
-  int lo = 0, hi = B - 1;
-  while (lo < hi) {  // last sequence whose first tile is <= tile
-    int mid = (lo + hi + 1) >> 1;
-    if (tile_off[mid] <= tile) lo = mid; else hi = mid - 1;
+  int seq, t0;
+  if (ml.fe_tiles != 0) {  // explicit tile list (resident stream windows: only some frames are recomputed)
+    seq = meta[ml.fe_tiles + 2 * blockIdx.x];
+    t0 = meta[ml.fe_tiles + 2 * blockIdx.x + 1];
+  } else {
+    const int* tile_off = meta + ml.fe_tile_off;
+    int tile = blockIdx.x;
+    int lo = 0, hi = B - 1;
+    while (lo < hi) {  // last sequence whose first tile is <= tile
+      int mid = (lo + hi + 1) >> 1;
+      if (tile_off[mid] <= tile) lo = mid; else hi = mid - 1;
+    }
+    seq = lo;
+    t0 = (tile - tile_off[seq]) * kFeFrames;
   }
-  const int seq = lo;
-  const int t0 = (tile - tile_off[seq]) * kFeFrames;
   const int T = meta[ml.frames + seq];
   const int s0 = meta[ml.sample_off + seq];
-  const int L_audio = meta[ml.sample_off + seq + 1] - s0;
+  const int L_audio = ml.fe_len != 0 ? meta[ml.fe_len + seq] : meta[ml.sample_off + seq + 1] - s0;
   const int L = L_audio + tail_len;  // the buffer followed by the raw-audio hush word, if any
   const float* x = audio + s0;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -218,6 +224,81 @@ void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, 
   if (n_tiles > 0)
     frontend_kernel<<<n_tiles, 256, smem, s>>>(audio, meta, ml, B, dft_basis, mel_fb_t, n_mel, logmel,
                                                 seq_max, tail, tail_len);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Resident stream windows (the audio buffer of a stream grows at its end every round and is cut
+// at its front now and then, Sec. 3.2): samples and un-normalised log-mel rows stay on the device
+// between rounds, and only the frames whose 400 samples changed are recomputed.
+
+// Drops `cut` floats at the front of a slice of `count` floats, in place.  One CTA per slice
+// walks it front to back; a chunk is read completely (into registers) before it is written, and
+// it is written to addresses below everything that is still to be read.
+constexpr int kShiftPerThread = 32;
+__global__ void __launch_bounds__(256) stream_shift_kernel(float* __restrict__ base_audio,
+                                                           float* __restrict__ base_logmel,
+                                                           const int* __restrict__ entries_audio,
+                                                           const int* __restrict__ entries_logmel) {
+  const int* en = (blockIdx.y == 0 ? entries_audio : entries_logmel) + 3 * blockIdx.x;
+  float* a = (blockIdx.y == 0 ? base_audio : base_logmel) + en[0];
+  const int cut = en[1], count = en[2];
+  if (cut <= 0) return;
+  const int keep = count - cut;
+  for (int c0 = 0; c0 < keep; c0 += 256 * kShiftPerThread) {
+    float v[kShiftPerThread];
+#pragma unroll
+    for (int u = 0; u < kShiftPerThread; ++u) {
+      const int i = c0 + u * 256 + threadIdx.x;
+      v[u] = i < keep ? a[cut + i] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < kShiftPerThread; ++u) {
+      const int i = c0 + u * 256 + threadIdx.x;
+      if (i < keep) a[i] = v[u];
+    }
+  }
+}
+
+void launch_stream_shift(float* base_audio, float* base_logmel, const int* entries_audio, const int* entries_logmel,
+                         int n, cudaStream_t s) {
+  if (n > 0) stream_shift_kernel<<<dim3(n, 2), 256, 0, s>>>(base_audio, base_logmel, entries_audio, entries_logmel);
+}
+
+__global__ void stream_append_kernel(float* __restrict__ audio, const float* __restrict__ new_audio,
+                                     const int* __restrict__ entries) {
+  const int* en = entries + 3 * blockIdx.y;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < en[2]) audio[en[0] + i] = new_audio[en[1] + i];
+}
+
+void launch_stream_append(float* audio, const float* new_audio, const int* entries, int n, int max_count,
+                          cudaStream_t s) {
+  if (n > 0 && max_count > 0)
+    stream_append_kernel<<<dim3((max_count + 255) / 256, n), 256, 0, s>>>(audio, new_audio, entries);
+}
+
+// 32 frames per CTA
+__global__ void __launch_bounds__(256) stream_max_kernel(const float* __restrict__ logmel,
+                                                         const int* __restrict__ meta, MetaLayout ml, int n_mel,
+                                                         int* __restrict__ seq_max) {
+  const int seq = blockIdx.y;
+  const int T = meta[ml.frames + seq];
+  const int t0 = blockIdx.x * 32;
+  if (t0 >= T) return;
+  const float* src = logmel + ((long)meta[ml.frame_off + seq] + t0) * n_mel;
+  const int count = min(32, T - t0) * n_mel;
+  float mx = -INFINITY;
+  for (int i = threadIdx.x; i < count; i += 256) mx = fmaxf(mx, src[i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((threadIdx.x & 31) == 0 && mx > -INFINITY) atomicMax(seq_max + seq, float_to_ordered(mx));
+}
+
+void launch_stream_max(const float* logmel, const int* meta, MetaLayout ml, int B, int max_frames, int n_mel,
+                       int* seq_max, cudaStream_t s) {
+  if (B > 0 && max_frames > 0)
+    stream_max_kernel<<<dim3((max_frames + 31) / 32, B), 256, 0, s>>>(logmel, meta, ml, n_mel, seq_max);
 }
 
 // ---------------------------------------------------------------------------------------------

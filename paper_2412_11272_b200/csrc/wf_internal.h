@@ -49,6 +49,10 @@ struct MetaLayout {
   int fe_tile_off;  // [B+1] prefix sums of front-end tiles
   int attn_work;    // [n_attn_work] pairs (sequence, first query row within the sequence)
   int total;
+  // front end over resident stream windows (0 = absent: lengths come from sample_off differences
+  // and tiles from fe_tile_off)
+  int fe_len;       // [B] samples in each buffer
+  int fe_tiles;     // [n_tiles] pairs (sequence, first frame of the tile)
 };
 
 // ---- kernel launch with optional cluster size and programmatic stream serialization.
@@ -101,6 +105,17 @@ void launch_normalise(const float* logmel, const int* seq_max, const float* mel_
 void launch_build_maps(const int* meta, MetaLayout ml, int B, int max_rows, int hush_frames,
                        int* row_valid, int2* row_dst, cudaStream_t s);
 void launch_fill_seq_max(int* seq_max, int B, cudaStream_t s);
+
+// ---- resident stream windows (wf_frontend.cu).  Lists live in one int buffer:
+// shift entries (float offset of the array slice, floats to drop at its front, floats in it),
+// append entries (destination float offset, source float offset, count).
+void launch_stream_shift(float* base_audio, float* base_logmel, const int* entries_audio, const int* entries_logmel,
+                         int n, cudaStream_t s);
+void launch_stream_append(float* audio, const float* new_audio, const int* entries, int n, int max_count,
+                          cudaStream_t s);
+// seq_max[i] = max over the frames[i] x n_mel values at logmel + frame_off[i] * n_mel (ordered ints)
+void launch_stream_max(const float* logmel, const int* meta, MetaLayout ml, int B, int max_frames, int n_mel,
+                       int* seq_max, cudaStream_t s);
 
 // ---- SIMT float32 kernels and element-wise kernels (wf_simt.cu)
 void launch_gemm_f32(const float* A, long lda, const float* W, long ldw, long M, int N, int K,

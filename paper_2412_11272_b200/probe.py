@@ -6,6 +6,7 @@
     python -m paper_2412_11272_b200.probe logmel --seconds 15 --batch 64
     python -m paper_2412_11272_b200.probe dtw --batch 64 --n 150
     python -m paper_2412_11272_b200.probe crosskv --M 49600 --layers 32
+    python -m paper_2412_11272_b200.probe streams --shape large --batch 64      (resident windows: push 1 s, encode, 15 rounds)
     python -m paper_2412_11272_b200.probe config --name small        (tiny, base, small, medium-padded, medium-hush, large)
 
 Each command warms up, times ``--iters`` launches with CUDA events on the launching stream and
@@ -21,7 +22,7 @@ import numpy as np
 import torch
 
 from . import inputs as I
-from .binding import Encoder
+from .binding import Encoder, Streams
 
 
 def _time(fn, iters, warmup=3):
@@ -44,7 +45,7 @@ def _component_encoder(d_model=128, n_head=2, max_batch=1, max_tokens=64):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["gemm", "attention", "encode", "logmel", "config", "dtw", "crosskv"])
+    ap.add_argument("what", choices=["gemm", "attention", "encode", "logmel", "config", "dtw", "crosskv", "streams"])
     ap.add_argument("--name", default="base")
     ap.add_argument("--M", type=int, default=16384)
     ap.add_argument("--N", type=int, default=3840)
@@ -88,6 +89,38 @@ def main():
         enc.wf_check()
         out.update(M=a.M, d_model=d, layers=a.layers, ms=ms, tflops=2.0 * a.M * N * d / ms / 1e9,
                    write_gbs=2.0 * a.M * N / ms / 1e6)
+    elif a.what == "streams":
+        # --batch streams, 15 rounds: every round each window grows by 1 s, then all windows are encoded;
+        # "push" times wf_streams_push (framing of the new second only), "front_end_full" times the
+        # front end over the whole windows (wf_logmel) for comparison
+        shape = I.SHAPES[a.shape]
+        B, rounds = a.batch, 15
+        tokens = int(I.tokens_of(np.full(B, rounds * 16000)).sum())
+        enc = Encoder(shape, I.encoder_weights(0, shape), I.mel_filterbank(shape.n_mel), B, tokens, B * rounds * 16000)
+        st = Streams(enc, B, rounds * 16000)
+        feed = torch.as_tensor(np.stack([I.synth_audio(0, b, rounds * 16000) for b in range(B)])).cuda()
+        hush = torch.as_tensor(I.round_to_bf16(I.hush_mel(0, shape.n_mel))).cuda()
+        outb = torch.empty((tokens, shape.d_model), dtype=enc.out_dtype, device="cuda")
+        ids = list(range(B))
+        ev = lambda: torch.cuda.Event(enable_timing=True)
+        push_ms = enc_ms = full_ms = 0.0
+        for k in range(1, rounds + 1):
+            new = feed[:, (k - 1) * 16000:k * 16000].contiguous().reshape(-1)
+            win = feed[:, :k * 16000].contiguous().reshape(-1)
+            e = [ev() for _ in range(4)]
+            e[0].record()
+            st.wf_streams_push(ids, new, [16000] * B)
+            e[1].record()
+            st.wf_encode_streams(ids, hush, out=outb)
+            e[2].record()
+            enc.wf_logmel(win, [k * 16000] * B)
+            e[3].record()
+            torch.cuda.synchronize()
+            push_ms += e[0].elapsed_time(e[1]); enc_ms += e[1].elapsed_time(e[2]); full_ms += e[2].elapsed_time(e[3])
+        enc.wf_check()
+        out.update(shape=a.shape, streams=B, rounds=rounds, push_ms_total=push_ms, encode_ms_total=enc_ms,
+                   front_end_full_ms_total=full_ms, audio_s_per_s=B * sum(range(1, rounds + 1)) / (push_ms + enc_ms) * 1e3)
+        st.close()
     elif a.what == "dtw":
         # --batch problems of --n tokens x (5 * --n) frames (150 tokens x 750 frames by default)
         n_tok, n_frm = (a.n if a.n != 775 else 150), 5 * (a.n if a.n != 775 else 150)

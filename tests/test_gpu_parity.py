@@ -399,6 +399,83 @@ def test_dtw_matches_oracle_bit_for_bit():
     enc.close()
 
 
+# ------------------------------------------------------------------------------ resident stream windows
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_stream_windows_match_encoding_from_scratch(dtype):
+    """Windows that grow at the end every round and are cut at the front now and then (Sec. 3.2):
+    only the changed frames are recomputed, and the encoding of the resident windows equals,
+    bit for bit, wf_encode of the same windows, and the oracle's from-scratch result."""
+    from paper_2412_11272_b200.binding import Streams, WfError
+    bf16 = dtype == "bf16"
+    shape = _small(dtype, n_layer=1, **({"d_model": 256, "n_head": 4, "d_mlp": 512} if bf16 else {}))
+    W = I.encoder_weights(21, shape)
+    hush_np = I.hush_mel(21, 80)
+    if bf16:
+        hush_np = I.round_to_bf16(hush_np)
+    hush = _dev(hush_np)
+    n_streams, cap = 4, 160 * 700
+    enc = make_encoder(shape, W, n_streams, 4 * 400, n_streams * cap)
+    st = Streams(enc, n_streams, cap)
+    feed = [I.synth_audio(21, 40 + i, 16000 * 12) for i in range(n_streams)]      # each stream's endless input
+    pos = [0] * n_streams                    # samples consumed from the feed
+    start = [0] * n_streams                  # first sample of the window within the feed
+    rng = np.random.default_rng(3)
+    for rnd in range(9):
+        ids = [i for i in range(n_streams) if rnd == 0 or rng.random() < 0.8] or [0]
+        ids = [int(i) for i in rng.permutation(ids)]
+        n_new, trim = [], []
+        for i in ids:
+            add = int(rng.choice([16000, 8000, 16000 + 37, 3 * 160 + 1, 700]))
+            win = pos[i] - start[i]
+            cut = 0
+            if rnd == 0:
+                add = max(add, 1000)
+            elif rnd == 7 and i == ids[0]:
+                cut, add = (win // 160) * 160, 16000                    # all but a ragged remainder goes
+            elif rnd in (3, 6) and win > 1200:
+                cut = 160 * int(rng.integers(1, (win - 800) // 160 + 1))
+            if win - cut + add > cap:
+                cut += -(-(win - cut + add - cap) // 160) * 160
+            n_new.append(add)
+            trim.append(cut)
+        new_audio = np.concatenate([feed[i][pos[i]:pos[i] + a] for i, a in zip(ids, n_new)])
+        st.wf_streams_push(ids, _dev(new_audio), n_new, trim)
+        for i, a, c in zip(ids, n_new, trim):
+            pos[i] += a
+            start[i] += c
+            assert st.wf_streams_length(i) == pos[i] - start[i]
+        live = [i for i in range(n_streams) if pos[i] - start[i] >= 401]
+        out, cu = st.wf_encode_streams(live, hush)
+        windows = [feed[i][start[i]:pos[i]] for i in live]
+        lengths = [len(w) for w in windows]
+        ref, cu_ref = enc.wf_encode(_dev(np.concatenate(windows)), lengths, hush)
+        enc.wf_check()
+        assert list(cu) == list(cu_ref)
+        assert torch.equal(out, ref), rnd
+        if rnd in (4, 8):
+            got = to_np(out)
+            for k, w in enumerate(windows[:2]):
+                r = O.encode_sequence(w, I.mel_filterbank(80), hush_np, W, shape.n_layer, shape.n_head)
+                if bf16:
+                    _check_bf16(got[cu[k]:cu[k + 1]], r)
+                else:
+                    assert np.max(np.abs(got[cu[k]:cu[k + 1]] - r)) <= F32_TOL
+    # errors leave the windows untouched
+    before = [st.wf_streams_length(i) for i in range(n_streams)]
+    for ids, n_new, trim, status in (([0, 0], [160, 160], None, "WF_ERR_INVALID_ARG"),
+                                     ([1], [160], [100], "WF_ERR_INVALID_ARG"),
+                                     ([1], [cap], None, "WF_ERR_CAPACITY"),
+                                     ([2], [0], [(before[2] // 160) * 160], "WF_ERR_TOO_SHORT"),
+                                     ([9], [160], None, "WF_ERR_INVALID_ARG")):
+        with pytest.raises(WfError) as ei:
+            st.wf_streams_push(ids, _dev(np.zeros(max(sum(n_new), 1), np.float32)), n_new, trim)
+        assert ei.value.status == status, (ids, n_new, trim)
+    assert [st.wf_streams_length(i) for i in range(n_streams)] == before
+    st.close()
+    enc.close()
+
+
 # ------------------------------------------------------------------------------ errors and edges
 
 def test_errors_and_edge_cases():
