@@ -1,0 +1,87 @@
+"""Randomised robustness sweep of the bf16 kernels: GEMM, variable-length attention and the whole
+encoder on shapes drawn around the tile and step boundaries.  Every launch is repeated and must
+reproduce its first result bit for bit (the default path has a fixed order of operations, so any
+difference is a data race), and is compared with a float32 evaluation on the device.  This is a
+race and edge-case detector; the parity claims are the oracle comparisons in the other files."""
+import math
+
+import numpy as np
+import pytest
+
+from paper_2412_11272_b200 import inputs as I
+from tests._util import make_encoder
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+D_MODEL, N_HEAD = 256, 4
+
+
+@pytest.fixture(scope="module")
+def enc():
+    shape = I.EncoderShape("sweep", 80, D_MODEL, 2, N_HEAD, 512, "bf16", n_ctx=1600)
+    e = make_encoder(shape, I.encoder_weights(3, shape), 24, 40000, 24 * 160 * 1500 + 1000)
+    yield e
+    e.close()
+
+
+def test_gemm_random_shapes(enc):
+    rng = np.random.default_rng(100)
+    for _ in range(120):
+        M = max(1, int(rng.choice([1, 7, 31, 127, 128, 129, 255, 257, 300, 1000, 4097, 9000, 20000])) + int(rng.integers(-3, 4)))
+        N, K, mode = 8 * int(rng.integers(1, 200)), 8 * int(rng.integers(1, 200)), int(rng.integers(0, 3))
+        A = torch.randn(M, K, device="cuda").to(torch.bfloat16)
+        W = (torch.randn(N, K, device="cuda") / math.sqrt(K)).to(torch.bfloat16)
+        b = torch.randn(N, device="cuda")
+        ref = A.float() @ W.float().T + b
+        outs = []
+        for _ in range(3):
+            if mode == 2:
+                C = torch.ones(M, N, device="cuda")
+                enc.wf_gemm_bf16(A, W, b, 2, C)
+                outs.append(C)
+            else:
+                outs.append(enc.wf_gemm_bf16(A, W, b, mode))
+        ref = ref + 1.0 if mode == 2 else torch.nn.functional.gelu(ref) if mode == 1 else ref
+        err = float(((outs[0].float() - ref).abs() / (ref.abs() + 1.0)).max())
+        assert all(torch.equal(outs[0], o) for o in outs[1:]), (M, N, K, mode)
+        assert err < (2e-4 * math.sqrt(K) if mode == 2 else 2.0 ** -7), (M, N, K, mode, err)
+    enc.wf_check()
+
+
+def test_attention_random_batches(enc):
+    rng = np.random.default_rng(101)
+    edges = [1, 2, 5, 31, 95, 96, 97, 127, 128, 129, 191, 192, 193, 255, 256, 257, 300, 513, 775, 1000, 1525]
+    for _ in range(120):
+        B = int(rng.integers(1, 20))
+        lens = [max(1, int(rng.choice(edges)) + int(rng.integers(-2, 3))) for _ in range(B)]
+        cu = np.concatenate([[0], np.cumsum(lens)])
+        qkv = (torch.randn(int(cu[-1]), 3 * D_MODEL, device="cuda") * float(rng.choice([0.5, 1.0, 3.0]))).to(torch.bfloat16)
+        outs = [enc.wf_attention(qkv, cu) for _ in range(3)]
+        assert all(torch.equal(outs[0], o) for o in outs[1:]), lens
+        q, k, v = qkv.float().split(D_MODEL, dim=1)
+        ref = torch.empty(int(cu[-1]), D_MODEL, device="cuda")
+        for i in range(B):
+            s, e = int(cu[i]), int(cu[i + 1])
+            qq, kk, vv = (t[s:e].view(-1, N_HEAD, 64).transpose(0, 1) for t in (q, k, v))
+            p = torch.softmax(qq @ kk.transpose(1, 2) / 8.0, dim=-1)
+            ref[s:e] = (p @ vv).transpose(0, 1).reshape(-1, D_MODEL)
+        assert float((outs[0].float() - ref).abs().max() / ref.abs().max()) < 4e-2, lens
+    enc.wf_check()
+
+
+def test_encode_random_batches_repeat_and_are_batch_invariant(enc):
+    rng = np.random.default_rng(102)
+    hush = torch.as_tensor(I.round_to_bf16(I.hush_mel(3, 80))).cuda()
+    for _ in range(60):
+        B = int(rng.integers(1, 24))
+        lens = np.array([int(rng.integers(401, 160 * 1500)) if rng.random() < 0.3
+                         else 160 * int(rng.integers(3, 400)) + int(rng.integers(0, 160)) for _ in range(B)])
+        batch = I.batch_from_lengths(int(rng.integers(0, 1000)), lens)
+        audio = torch.as_tensor(batch.audio).cuda()
+        outs = [enc.wf_encode(audio, batch.lengths, hush)[0] for _ in range(3)]
+        assert all(torch.equal(outs[0], o) for o in outs[1:]), list(lens)
+        assert bool(torch.isfinite(outs[0].float()).all())
+        solo = enc.wf_encode(audio[:int(lens[0])].contiguous(), lens[:1], hush)[0]     # sequence 0 alone
+        assert float((solo.float() - outs[0][:solo.shape[0]].float()).abs().max()) < 0.1, list(lens)
+    enc.wf_check()
