@@ -98,7 +98,7 @@ struct Plan {
   int B;
   long total_samples;
   int total_frames, total_prows, total_tokens;
-  int n_fe_tiles, n_work, n_work_b, max_prows_seq;
+  int n_fe_tiles, n_work, n_attn_items, max_prows_seq;
   MetaLayout ml;
 };
 
@@ -178,14 +178,17 @@ class Prof {
   ProfEvent* ev_;
 };
 
-// Attention work list for sequences in `order` (tok[i] .. tok[i+1] are sequence i's tokens), as
-// (sequence, first query row) pairs written at `dst`.  float32 kernel: one entry per 16 rows.
-// bf16 kernel: first the entries of 256 consecutive rows whose two 128-row tiles are both
-// non-empty (*n_a of them), then one entry for the odd last tile of every sequence that has one
-// (*n_b; those run two heads side by side).
-void build_attn_work(const int* tok, const std::vector<int>& order, bool bf16, int* dst, int* n_a, int* n_b) {
+// Attention work list for sequences in `order` (tok[i] .. tok[i+1] are sequence i's tokens), written
+// at `dst`; returns the number of ints written.  float32 kernel: (sequence, first query row) pairs,
+// one per 16 rows, *n_entries of them.  bf16 kernel: (sequence, first query row | kind << 30, first
+// item) triples: per sequence the entries of 256 consecutive rows whose two 128-row tiles are both
+// non-empty (kind 0, n_head items each), then one entry for its odd last tile if it has one
+// (kind 1, two heads side by side: ceil(n_head / 2) items), then one int per item naming its entry.
+// *n_items counts the bf16 items.
+int build_attn_work(const int* tok, const std::vector<int>& order, bool bf16, int n_head, int* dst, int* n_entries,
+                    int* n_items) {
   int nw = 0;
-  *n_b = 0;
+  *n_items = 0;
   if (!bf16) {
     for (int i : order)
       for (int q0 = 0; q0 < tok[i + 1] - tok[i]; q0 += 16) {
@@ -193,25 +196,37 @@ void build_attn_work(const int* tok, const std::vector<int>& order, bool bf16, i
         dst[2 * nw + 1] = q0;
         ++nw;
       }
-    *n_a = nw;
-    return;
+    *n_entries = nw;
+    return 2 * nw;
   }
-  for (int i : order)
-    for (int q0 = 0; q0 + 128 < tok[i + 1] - tok[i]; q0 += 256) {
-      dst[2 * nw] = i;
-      dst[2 * nw + 1] = q0;
-      ++nw;
-    }
-  *n_a = nw;
+  int items = 0;
   for (int i : order) {
-    const int tiles = (tok[i + 1] - tok[i] + 127) / 128;
-    if (tiles & 1) {
-      dst[2 * nw] = i;
-      dst[2 * nw + 1] = (tiles - 1) * 128;
+    const int n = tok[i + 1] - tok[i];
+    for (int q0 = 0; q0 + 128 < n; q0 += 256) {
+      dst[3 * nw] = i;
+      dst[3 * nw + 1] = q0;
+      dst[3 * nw + 2] = items;
+      items += n_head;
       ++nw;
-      ++*n_b;
+    }
+    const int tiles = (n + 127) / 128;
+    if (tiles & 1) {
+      dst[3 * nw] = i;
+      dst[3 * nw + 1] = ((tiles - 1) * 128) | (1 << 30);
+      dst[3 * nw + 2] = items;
+      items += (n_head + 1) / 2;
+      ++nw;
     }
   }
+  *n_entries = nw;
+  *n_items = items;
+  // one int per item: the entry it belongs to (saves the kernel a search)
+  int* item_entry = dst + 3 * nw;
+  for (int w = 0; w < nw; ++w) {
+    const int end = w + 1 < nw ? dst[3 * (w + 1) + 2] : items;
+    for (int it = dst[3 * w + 2]; it < end; ++it) item_entry[it] = w;
+  }
+  return 3 * nw + items;
 }
 
 // Builds prefix sums, the padded-row layout and the work lists for one call into `hm`
@@ -274,9 +289,9 @@ wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Pl
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
     return hm[ml.tok_off + a + 1] - hm[ml.tok_off + a] > hm[ml.tok_off + b + 1] - hm[ml.tok_off + b];
   });
-  int nw = 0, nw_b = 0;
-  if (build_work) build_attn_work(hm + ml.tok_off, order, e->bf16, hm + ml.attn_work, &nw, &nw_b);
-  ml.total = ml.attn_work + 2 * (nw + nw_b);
+  int nw = 0, n_items = 0, work_ints = 0;
+  if (build_work) work_ints = build_attn_work(hm + ml.tok_off, order, e->bf16, c.n_head, hm + ml.attn_work, &nw, &n_items);
+  ml.total = ml.attn_work + work_ints;
   p->B = B;
   p->total_samples = samples;
   p->total_frames = (int)frames;
@@ -284,7 +299,7 @@ wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Pl
   p->total_tokens = (int)tokens;
   p->n_fe_tiles = (int)tiles;
   p->n_work = nw;
-  p->n_work_b = nw_b;
+  p->n_attn_items = n_items;
   p->max_prows_seq = max_pr;
   return WF_OK;
 }
@@ -354,7 +369,7 @@ wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidde
     }
     {
       Prof pr(e, 5, s);
-      if (e->bf16) launch_attention_bf16(e->tm_qkv, e->tm_qkv_kv, (__nv_bfloat16*)e->attn, meta, p.ml, p.n_work, p.n_work_b, d, e->err_flag, e->num_sms, s);
+      if (e->bf16) launch_attention_bf16(e->tm_qkv, e->tm_qkv_kv, (__nv_bfloat16*)e->attn, meta, p.ml, p.n_work, p.n_attn_items, d, e->err_flag, e->num_sms, s);
       else launch_attention_f32((const float*)e->qkv, (float*)e->attn, meta, p.ml, p.n_work, d, s);
     }
     {
@@ -547,7 +562,8 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
   WF_TRY(dev_alloc<float>(e, &e->audio_stage, (size_t)c.max_samples));
   WF_TRY(dev_alloc_bytes(e, &e->out_stage, mt * d * e->esz));
   WF_TRY(dev_alloc<int>(e, &e->err_flag, 1, true));
-  e->meta_cap = 6 * (c.max_batch + 1) + 2 * (int)(c.max_tokens / 16 + c.max_batch) + 16;
+  e->meta_cap = 6 * (c.max_batch + 1) + 2 * (int)(c.max_tokens / 16 + c.max_batch) + 6 * c.max_batch + 16 +
+                (e->bf16 ? (int)(c.max_tokens / 256 + 2 * c.max_batch) * c.n_head : 0);
   for (int i = 0; i < kRing; ++i) {
     WF_TRY(dev_alloc<int>(e, &e->meta_dev[i], e->meta_cap));
     void* hp = nullptr;
@@ -1023,9 +1039,8 @@ wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, in
   for (int i = 0; i <= B; ++i) hm[i] = cu_seqlens[i];
   std::vector<int> order(B);
   for (int i = 0; i < B; ++i) order[i] = i;
-  int nw = 0, nw_b = 0;
-  build_attn_work(hm, order, e->bf16, hm + ml.attn_work, &nw, &nw_b);
-  ml.total = ml.attn_work + 2 * (nw + nw_b);
+  int nw = 0, n_items = 0;
+  ml.total = ml.attn_work + build_attn_work(hm, order, e->bf16, e->cfg.n_head, hm + ml.attn_work, &nw, &n_items);
   Plan p{};
   p.ml = ml;
   st = ring_upload(e, slot, p, s);
@@ -1037,7 +1052,7 @@ wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, in
       if (!make_tmap_bf16(e->tma, &tq, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 128) ||
           !make_tmap_bf16(e->tma, &tkv, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 96))
         return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected the qkv tensor map");
-      launch_attention_bf16(tq, tkv, (__nv_bfloat16*)out, e->meta_dev[slot], ml, nw, nw_b, e->cfg.d_model, e->err_flag, e->num_sms, s);
+      launch_attention_bf16(tq, tkv, (__nv_bfloat16*)out, e->meta_dev[slot], ml, nw, n_items, e->cfg.d_model, e->err_flag, e->num_sms, s);
     }
     else launch_attention_f32((const float*)qkv, (float*)out, e->meta_dev[slot], ml, nw, e->cfg.d_model, s);
   }

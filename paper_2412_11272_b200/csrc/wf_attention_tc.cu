@@ -71,27 +71,28 @@ struct Item {
   bool split;  // the tiles belong to different heads: K / V stages alternate between them
 };
 
-// Items [0, n_work_a * n_head): work entry = 256 consecutive rows (both tiles non-empty), one item
-// per head.  The rest: work entry = the odd last tile of a sequence, one item per pair of heads
-// (a last unpaired head runs as a single tile).
+// The work list holds (sequence, first query row | kind << 30, first item) triples in launch order;
+// kind 0: 256 consecutive rows (both tiles non-empty), one item per head; kind 1: the odd last
+// tile of a sequence, one item per pair of heads (a last unpaired head runs as a single tile).
+// An entry of kind 1 directly follows the other entries of its sequence, so that its K / V tiles
+// are still in the L2 when it runs.  Behind the triples sits one int per item: its entry.
 __device__ __forceinline__ Item load_item(const int* __restrict__ meta, const MetaLayout& ml, int it, int n_head,
-                                          int n_work_a) {
+                                          int n_entries) {
+  const int* wl = meta + ml.attn_work;
+  const int lo = wl[3 * n_entries + it];  // the entry of every item follows the triples
+  const int local = it - wl[3 * lo + 2];
+  const int seq = wl[3 * lo], q0k = wl[3 * lo + 1];
   Item w;
-  int work;
-  if (it < n_work_a * n_head) {
-    work = it / n_head;
-    w.head = w.head1 = it - work * n_head;
+  w.q0 = q0k & 0x3FFFFFFF;
+  if ((q0k >> 30) == 0) {
+    w.head = w.head1 = local;
     w.two = true;
     w.split = false;
   } else {
-    const int itb = it - n_work_a * n_head, hp = (n_head + 1) >> 1;
-    work = n_work_a + itb / hp;
-    w.head = 2 * (itb % hp);
+    w.head = 2 * local;
     w.two = w.split = w.head + 1 < n_head;
     w.head1 = w.two ? w.head + 1 : w.head;
   }
-  const int seq = meta[ml.attn_work + 2 * work];
-  w.q0 = meta[ml.attn_work + 2 * work + 1];
   w.q1 = w.split ? w.q0 : w.q0 + kTQ;
   w.tok0 = meta[ml.tok_off + seq];
   w.n = meta[ml.tok_off + seq + 1] - w.tok0;
@@ -103,7 +104,7 @@ __device__ __forceinline__ Item load_item(const int* __restrict__ meta, const Me
 
 __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
     const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
-    __nv_bfloat16* __restrict__ out, const int* __restrict__ meta, MetaLayout ml, int n_items, int n_work_a,
+    __nv_bfloat16* __restrict__ out, const int* __restrict__ meta, MetaLayout ml, int n_items, int n_entries,
     int n_head, int d_model, int* err_flag) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -163,7 +164,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
       uint32_t kc = 0, vc = 0, items = 0;
       bool ok = true;
       for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-        const Item w = load_item(meta, ml, it, n_head, n_work_a);
+        const Item w = load_item(meta, ml, it, n_head, n_entries);
         if (!mbar_wait(q_free, (items & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         mbar_arrive_expect_tx(q_full, w.two ? 2 * kQBytes : kQBytes);
         tma_load_2d(sbase + kOffQ, &tmap_q, w.head * kHeadDim, w.tok0 + w.q0, q_full);
@@ -228,7 +229,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
       __syncwarp();
     };
     for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-      const Item w = load_item(meta, ml, it, n_head, n_work_a);
+      const Item w = load_item(meta, ml, it, n_head, n_entries);
       if (t == 1 && !w.two) {
         // nothing to compute for this tile: release the stages in step with the other tile
         for (int j = 0; ok && j < w.n_kv; ++j) {
@@ -319,7 +320,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
     };
 
     for (int it = blockIdx.x; ok && it < n_items; it += gridDim.x) {
-      const Item w = load_item(meta, ml, it, n_head, n_work_a);
+      const Item w = load_item(meta, ml, it, n_head, n_entries);
       if (t == 1 && !w.two) continue;
       // a warp whose 32 rows all lie beyond the sequence keeps pace with the barriers only
       const int row0 = t ? w.q1 : w.q0;  // first query row of this tile
@@ -462,14 +463,13 @@ cudaError_t attention_bf16_configure() {
 }
 
 void launch_attention_bf16(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, __nv_bfloat16* out,
-                           const int* meta, MetaLayout ml, int n_work_a, int n_work_b, int d_model, int* err_flag,
+                           const int* meta, MetaLayout ml, int n_entries, int n_items, int d_model, int* err_flag,
                            int num_sms, cudaStream_t s) {
-  const int n_head = d_model / kHeadDim;
-  const int n_items = n_work_a * n_head + n_work_b * ((n_head + 1) / 2);
   if (n_items <= 0) return;
+  const int n_head = d_model / kHeadDim;
   const int grid = n_items < num_sms ? n_items : num_sms;
   launch_dependent(attention_tc_kernel, dim3(grid), dim3(kAttnThreads), kAttnSmem, s, 1, tmap_q, tmap_kv, out, meta, ml,
-                   n_items, n_work_a, n_head, d_model, err_flag);
+                   n_items, n_entries, n_head, d_model, err_flag);
 }
 
 }  // namespace wf

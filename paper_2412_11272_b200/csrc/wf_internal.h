@@ -157,13 +157,14 @@ void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtens
                       int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s);
 
 // ---- bf16 attention on tcgen05 (wf_attention_tc.cu).  The work list at ml.attn_work holds
-// n_work_a entries of 256 consecutive query rows (one item per head) followed by n_work_b
-// entries naming the odd last 128-row tile of a sequence (one item per pair of heads).
+// n_entries triples (sequence, first query row | kind << 30, first item): kind 0 = 256 consecutive
+// query rows, one item per head; kind 1 = the odd last 128-row tile of a sequence, one item per
+// pair of heads; behind the triples one int per item names its entry.  n_items is the total.
 cudaError_t attention_bf16_configure();
 // tmap_q / tmap_kv: bf16 [rows, 3 d_model] maps of the same buffer with 64 x 128 and 64 x 96 boxes
 // (make_tmap_bf16 with box_rows 128 and 96)
 void launch_attention_bf16(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, __nv_bfloat16* out,
-                           const int* meta, MetaLayout ml, int n_work_a, int n_work_b, int d_model, int* err_flag,
+                           const int* meta, MetaLayout ml, int n_entries, int n_items, int d_model, int* err_flag,
                            int num_sms, cudaStream_t s);
 
 // ---- dynamic time warping (wf_dtw.cu); meta holds 4 ints per problem:
