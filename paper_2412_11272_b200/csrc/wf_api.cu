@@ -496,6 +496,8 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     // to run, so results are no longer bit-reproducible).  Off unless asked for.
     const char* pdl_env = getenv("WF_PDL");
     pdl_set(!(pdl_env != nullptr && pdl_env[0] == '0'));
+    const char* small_env = getenv("WF_GEMM_SMALL_TILES");
+    gemm_bf16_set_small_tiles(!(small_env != nullptr && small_env[0] == '0'));
     const char* split_env = getenv("WF_GEMM_TAIL_SPLIT");
     gemm_bf16_set_tail_split(split_env != nullptr && split_env[0] == '1');
   }

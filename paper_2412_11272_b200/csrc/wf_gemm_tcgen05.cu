@@ -544,6 +544,9 @@ cudaError_t gemm_bf16_configure() {
   if ((e = configure_one<256, kEpiBiasResid>()) != cudaSuccess) return e;
   if ((e = configure_one<256, kEpiConv1>()) != cudaSuccess) return e;
   if ((e = configure_one<256, kEpiConv2>()) != cudaSuccess) return e;
+  if ((e = configure_one<128, kEpiBias>()) != cudaSuccess) return e;
+  if ((e = configure_one<128, kEpiBiasGelu>()) != cudaSuccess) return e;
+  if ((e = configure_one<128, kEpiBiasResid>()) != cudaSuccess) return e;
   return cudaSuccess;
 }
 
@@ -559,9 +562,11 @@ static void launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUten
 // pair = 1: CTA-pair kernel (W maps must then use 128-row boxes); 0: single-CTA kernel
 static int g_gemm_use_pair = 1;
 static int g_gemm_tail_split = 0;
+static int g_gemm_small_tiles = 1;
 void gemm_bf16_set_pair(int on) { g_gemm_use_pair = on; }
 int gemm_bf16_uses_pair() { return g_gemm_use_pair; }
 void gemm_bf16_set_tail_split(int on) { g_gemm_tail_split = on; }
+void gemm_bf16_set_small_tiles(int on) { g_gemm_small_tiles = on; }
 
 template <int EPI>
 static void launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
@@ -587,6 +592,27 @@ void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtens
                       int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
   if (M <= 0 || N <= 0 || K <= 0) return;
   if (g_gemm_use_pair) {
+    // Small problems leave most CTA pairs idle or waste most of a last round of 256 x 256 tiles:
+    // 128 x 128 tiles on single CTAs (same tensor maps: both use 128-row boxes) quarter the
+    // granularity.  Estimated rounds, a 128 x 128 tile counted as half a pair tile's time times
+    // kSmallTilePenalty for its lower efficiency (it reads shared memory at the full 128 B/clk;
+    // measured: a round of small tiles takes ~0.8 of a round of pair tiles).
+    if (g_gemm_small_tiles && epi <= kEpiBiasResid && a_cols == K) {
+      constexpr double kSmallTilePenalty = 1.6;
+      const long t_pair = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + 255) / 256);
+      const long t_small = ((M + kBM - 1) / kBM) * ((N + 127) / 128);
+      const long n_pairs = num_sms / 2;
+      const double r_pair = (double)((t_pair + n_pairs - 1) / n_pairs);
+      const double r_small = (double)((t_small + num_sms - 1) / num_sms) * 0.5 * kSmallTilePenalty;
+      if (r_small < r_pair) {
+        switch (epi) {
+          case kEpiBias: launch_one<128, kEpiBias>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+          case kEpiBiasGelu: launch_one<128, kEpiBiasGelu>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+          default: launch_one<128, kEpiBiasResid>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+        }
+        return;
+      }
+    }
     switch (epi) {
       case kEpiBias: launch_pair<kEpiBias>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
       case kEpiBiasGelu: launch_pair<kEpiBiasGelu>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;

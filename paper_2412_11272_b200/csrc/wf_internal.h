@@ -148,6 +148,8 @@ void gemm_bf16_set_pair(int on);
 // 1: residual-epilogue GEMMs cut the tiles of their last, partial round along K (default 0:
 // the order of the float32 residual additions, and with it every output bit, is then fixed)
 void gemm_bf16_set_tail_split(int on);
+// 1 (default): GEMMs too small to fill the CTA pairs with 256 x 256 tiles run 128 x 128 tiles on single CTAs
+void gemm_bf16_set_small_tiles(int on);
 // a_cols: stored row length of A in elements (K for a plain GEMM; smaller when one GEMM row
 // spans several consecutive stored rows, which must then be a multiple of 64).
 // tc: output map (bf16 out for kEpiBias/kEpiBiasGelu/kEpiConv1, float32 residual for
