@@ -81,7 +81,16 @@ typedef struct {
  * read, builds the windowed-DFT and sinusoid tables on the device, allocates workspace for
  * the stated capacities.  Synchronises `stream` before returning.  Fails with
  * WF_ERR_UNSUPPORTED_ARCH on a device that is not compute capability 10.x.
- * (Operation: the encoder of Sec. 1.1 / Sec. 2.3; weights are caller-provided.) */
+ * (Operation: the encoder of Sec. 1.1 / Sec. 2.3; weights are caller-provided.)
+ * Three process-wide tuning switches of the WF_BF16 path are read from the environment here:
+ *   WF_PDL=0               launch kernels plainly instead of with programmatic stream
+ *                          serialization (on by default: a kernel's set-up overlaps the tail of
+ *                          the kernel before it);
+ *   WF_GEMM_SMALL_TILES=0  never use 128 x 128 single-CTA tiles for small GEMMs;
+ *   WF_GEMM_TAIL_SPLIT=1   cut the last partial round of a residual GEMM's tiles along K (faster
+ *                          at small M; results then vary in the last bit from run to run, which
+ *                          is why it is off by default).
+ * None of them changes what is computed beyond float32 rounding order. */
 wf_status wf_encoder_create(const wf_config *cfg, const wf_weights *w, void *stream,
                             wf_encoder **out);
 
