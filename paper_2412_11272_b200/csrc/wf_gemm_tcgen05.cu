@@ -79,7 +79,7 @@ __device__ __forceinline__ void conv2_store32(const EpiParams& ep, long row, lon
 // Epilogue of one 128 x BN accumulator tile for the warp that owns TMEM lanes 32 * quarter ..:
 // t_row is the tensor-memory address of that lane group's first column of the tile, m0 / n0 the
 // tile origin in the output, stage_base this warp's two 4 KB staging buffers.
-template <int BN, int EPI>
+template <int BN, int EPI, int NBUF = 2>
 __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtensorMap* tmap_c, uint32_t t_row, int m0,
                                               int n0, long M, int N, int quarter, int lane, uint32_t stage_base,
                                               uint32_t& piece, bool with_bias = true) {
@@ -98,8 +98,8 @@ __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtenso
     // float32: 32 columns = 128 bytes per row and piece
 #pragma unroll 1
     for (int c = 0; c < BN / 32; ++c) {
-      const uint32_t buf = stage_base + (uint32_t)((piece & 1) * 4096);
-      if (lane == 0) bulk_wait_read<1>();   // the copy that last read this buffer is done with it
+      const uint32_t buf = stage_base + (uint32_t)((piece % NBUF) * 4096);
+      if (lane == 0) bulk_wait_read<NBUF - 1>();   // the copy that last read this buffer is done with it
       __syncwarp();
       uint32_t a32[32];
       float v[32];
@@ -125,8 +125,8 @@ __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtenso
     if (EPI == kEpiConv1) valid = row < M && ep.row_valid[row] != 0;
 #pragma unroll 1
     for (int c = 0; c < BN / 64; ++c) {
-      const uint32_t buf = stage_base + (uint32_t)((piece & 1) * 4096);
-      if (lane == 0) bulk_wait_read<1>();
+      const uint32_t buf = stage_base + (uint32_t)((piece % NBUF) * 4096);
+      if (lane == 0) bulk_wait_read<NBUF - 1>();
       __syncwarp();
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
@@ -337,12 +337,17 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
     const __grid_constant__ CUtensorMap tmap_c, long M, int N, int K, int a_cols, EpiParams ep, int* err_flag,
     int tail_split) {
   constexpr int BN = 256;
-  constexpr int kStages = 6;
+  // The float32 add-reduction holds its staging buffer for ~2 us (the L2 performs the additions), so
+  // with two buffers per warp the residual epilogue is latency-bound at ~13 GB/s per CTA and the
+  // K = 1280 out-projection waits for it: that epilogue gets four buffers per warp, paid for with
+  // one operand stage.
+  constexpr int kStages = EPI == kEpiBiasResid ? 5 : 6;
+  constexpr int kBufs = EPI == kEpiBiasResid ? 4 : 2;
   constexpr int kABytes = kBM * kBK * 2;          // this CTA's 128 rows of A
   constexpr int kBBytes = (BN / 2) * kBK * 2;     // this CTA's 128 of the 256 W rows
   constexpr int kStageBytes = kABytes + kBBytes;  // 32 KB
   constexpr int kStagingOffset = kStages * kStageBytes;
-  constexpr int kBarOffset = kStagingOffset + 4 * 2 * 4096;
+  constexpr int kBarOffset = kStagingOffset + 4 * kBufs * 4096;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -445,7 +450,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
     }
   } else {
     const int quarter = warp & 3;
-    const uint32_t stage_base = smem_base + kStagingOffset + (uint32_t)((warp - 2) * 8192);
+    const uint32_t stage_base = smem_base + kStagingOffset + (uint32_t)((warp - 2) * kBufs * 4096);
     uint32_t piece = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -460,7 +465,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
         break;
       }
       tc_fence_after();
-      epilogue_tile<BN, EPI>(ep, &tmap_c, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN), m0, n0,
+      epilogue_tile<BN, EPI, kBufs>(ep, &tmap_c, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN), m0, n0,
                              M, N, quarter, lane, stage_base, piece, w.first);
       tc_fence_before();
       __syncwarp();
