@@ -340,6 +340,28 @@ def test_bf16_small_ragged_matches_oracle():
     enc.close()
 
 
+def test_bf16_many_minimal_buffers():
+    """400 buffers, most of them the shortest the front end accepts (401 samples: 2 frames + hush =
+    26 tokens), some a little longer: work lists, tile maps and metadata at a high sequence count."""
+    shape = _small("bf16", d_model=256, n_head=4, d_mlp=512, n_layer=2)
+    W = I.encoder_weights(12, shape)
+    rng = np.random.default_rng(12)
+    lengths = [401 if rng.random() < 0.7 else int(rng.integers(402, 160 * 12)) for _ in range(400)]
+    batch = I.batch_from_lengths(13, lengths)
+    hush = I.round_to_bf16(I.hush_mel(13, shape.n_mel))
+    tokens = int(I.tokens_of(batch.lengths).sum())
+    enc = make_encoder(shape, W, 400, tokens, int(batch.lengths.sum()))
+    out, cu = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush))
+    again, _ = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush))
+    enc.wf_check()
+    assert cu[-1] == tokens and torch.equal(out, again)
+    got = to_np(out)
+    picks = [0, 1, 199, 398, 399, int(np.argmax(lengths))]
+    for i, r in oracle_hidden(batch, shape, W, hush, only=set(picks)).items():
+        _check_bf16(got[cu[i]:cu[i + 1]], r)
+    enc.close()
+
+
 def test_bf16_attention_stress_weights():
     """Query/key weights scaled so that logits have a standard deviation of a few units."""
     shape = _small("bf16", d_model=256, n_head=4, d_mlp=512, n_layer=2)
