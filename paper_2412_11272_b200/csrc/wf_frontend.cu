@@ -5,6 +5,7 @@
 // All arithmetic is float32: the clamp at (max - 8) exposes 80 dB of dynamic range, which
 // bfloat16 products cannot resolve.
 #include "wf_internal.h"
+#include "wf_ptx.cuh"
 
 namespace wf {
 
@@ -70,6 +71,8 @@ void launch_fill_seq_max(int* seq_max, int B, cudaStream_t s) {
 // 8-frame x 7-bin register tile per thread; phase 3 squares into shared memory; phase 4 is
 // the mel projection, log10 and the per-buffer running maximum.
 constexpr int kPStride = 204;
+constexpr int kBasisChunk = 8;  // folded-DFT rows per staged chunk (a multiple of 4 that divides 200)
+constexpr int kFeSmemFloats = kFeFrames * kPStride > 2 * kFeFrames * kFold ? kFeFrames * kPStride : 2 * kFeFrames * kFold;
 
 __global__ void __launch_bounds__(256) frontend_kernel(
     const float* __restrict__ audio, const int* __restrict__ meta, MetaLayout ml, int B,
@@ -79,6 +82,7 @@ __global__ void __launch_bounds__(256) frontend_kernel(
   float* e_s = smem;                       // [64][200]
   float* o_s = smem + kFeFrames * kFold;   // [64][200]
   float* p_s = smem;                       // [64][204] after the DFT
+  float* b_s = smem + kFeSmemFloats;       // [2 buffers][cos, sin][kBasisChunk][224] staged basis rows
 
   int seq, t0;
   if (ml.fe_tiles != 0) {  // explicit tile list (resident stream windows: only some frames are recomputed)
@@ -128,36 +132,64 @@ __global__ void __launch_bounds__(256) frontend_kernel(
 #pragma unroll
     for (int j = 0; j < 7; ++j) { acc_r[f][j] = 0.f; acc_i[f][j] = 0.f; }
 
-  const float* bc = basis + lane;
-  const float* bs = basis + kFold * kBasisCols + lane;
+  // The cosine / sine rows are staged through shared memory kBasisChunk at a time (cp.async, double
+  // buffered): all eight warps read the same rows, and fetching them per warp through the L1 made
+  // this loop wait on the L1 rather than on the FMA pipe.
+  auto stage_basis = [&](int chunk, int buf) {
+    float* dst = b_s + buf * (2 * kBasisChunk * kBasisCols);
+    const int rows = min(kBasisChunk, kFold - chunk * kBasisChunk);
+    const int vec_per_half = rows * kBasisCols / 4;  // 16-byte pieces of the cosine (or sine) rows
+    for (int v = tid; v < 2 * vec_per_half; v += 256) {
+      const int half = v >= vec_per_half ? 1 : 0, idx = v - half * vec_per_half;
+      ptx::cp_async_16(ptx::smem_u32(dst + half * kBasisChunk * kBasisCols + 4 * idx),
+                       basis + (size_t)half * kFold * kBasisCols + (size_t)chunk * kBasisChunk * kBasisCols + 4 * idx,
+                       true);
+    }
+    ptx::cp_async_commit();
+  };
   const float* er = e_s + warp * 8 * kFold;
   const float* orow = o_s + warp * 8 * kFold;
-  for (int n4 = 0; n4 < kFold; n4 += 4) {
-    float4 ev[8], ov[8];
-#pragma unroll
-    for (int f = 0; f < 8; ++f) {
-      ev[f] = *reinterpret_cast<const float4*>(er + f * kFold + n4);
-      ov[f] = *reinterpret_cast<const float4*>(orow + f * kFold + n4);
+  constexpr int kChunks = (kFold + kBasisChunk - 1) / kBasisChunk;
+  stage_basis(0, 0);
+  for (int ch = 0; ch < kChunks; ++ch) {
+    if (ch + 1 < kChunks) {
+      stage_basis(ch + 1, (ch + 1) & 1);
+      ptx::cp_async_wait<1>();
+    } else {
+      ptx::cp_async_wait<0>();
     }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      float c[7], s[7];
-#pragma unroll
-      for (int j = 0; j < 7; ++j) {
-        c[j] = __ldg(bc + (n4 + u) * kBasisCols + 32 * j);
-        s[j] = __ldg(bs + (n4 + u) * kBasisCols + 32 * j);
-      }
+    __syncthreads();  // chunk ch has landed for every thread
+    const float* bc = b_s + (ch & 1) * (2 * kBasisChunk * kBasisCols) + lane;
+    const float* bs = bc + kBasisChunk * kBasisCols;
+    const int n_lo = ch * kBasisChunk, n_hi = min(kFold, n_lo + kBasisChunk);
+    for (int n4 = n_lo; n4 < n_hi; n4 += 4) {
+      float4 ev[8], ov[8];
 #pragma unroll
       for (int f = 0; f < 8; ++f) {
-        float e = u == 0 ? ev[f].x : u == 1 ? ev[f].y : u == 2 ? ev[f].z : ev[f].w;
-        float o = u == 0 ? ov[f].x : u == 1 ? ov[f].y : u == 2 ? ov[f].z : ov[f].w;
+        ev[f] = *reinterpret_cast<const float4*>(er + f * kFold + n4);
+        ov[f] = *reinterpret_cast<const float4*>(orow + f * kFold + n4);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        float c[7], s[7];
 #pragma unroll
         for (int j = 0; j < 7; ++j) {
-          acc_r[f][j] = fmaf(e, c[j], acc_r[f][j]);
-          acc_i[f][j] = fmaf(o, s[j], acc_i[f][j]);
+          c[j] = bc[(n4 - n_lo + u) * kBasisCols + 32 * j];
+          s[j] = bs[(n4 - n_lo + u) * kBasisCols + 32 * j];
+        }
+#pragma unroll
+        for (int f = 0; f < 8; ++f) {
+          float e = u == 0 ? ev[f].x : u == 1 ? ev[f].y : u == 2 ? ev[f].z : ev[f].w;
+          float o = u == 0 ? ov[f].x : u == 1 ? ov[f].y : u == 2 ? ov[f].z : ov[f].w;
+#pragma unroll
+          for (int j = 0; j < 7; ++j) {
+            acc_r[f][j] = fmaf(e, c[j], acc_r[f][j]);
+            acc_i[f][j] = fmaf(o, s[j], acc_i[f][j]);
+          }
         }
       }
     }
+    __syncthreads();  // everyone is done with this buffer before chunk ch + 2 overwrites it
   }
   __syncthreads();  // every warp is done with e_s / o_s before p_s overwrites them
 #pragma unroll
@@ -214,8 +246,7 @@ __global__ void __launch_bounds__(256) frontend_kernel(
 void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, int n_tiles,
                      const float* dft_basis, const float* mel_fb_t, int n_mel, float* logmel,
                      int* seq_max, const float* tail, int tail_len, cudaStream_t s) {
-  const int smem = (kFeFrames * kPStride > 2 * kFeFrames * kFold ? kFeFrames * kPStride : 2 * kFeFrames * kFold) *
-                   (int)sizeof(float);  // 102,400 B
+  const int smem = (kFeSmemFloats + 2 * 2 * kBasisChunk * kBasisCols) * (int)sizeof(float);  // 102,400 + 28,672 B
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(frontend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
