@@ -28,6 +28,8 @@
 // sequence is masked in the softmax, so no padded token ever contributes.
 // Tensor-memory columns per query tile t (base 256 t): S [0,96) f32; P0 [96,144), P1 [144,192)
 // packed bf16; O [192,256) f32.  Every mbarrier wait is bounded (wf_ptx.cuh).
+#include <type_traits>
+
 #include "wf_internal.h"
 #include "wf_ptx.cuh"
 
@@ -386,14 +388,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
           // behind S tracks every earlier MMA of that thread: having seen s_full, it has landed.
           float rs = 0.f, rs1 = 0.f;
           const uint32_t ta_p = ta_s + 96 + 48 * (g & 1u);
-#pragma unroll
-          for (int h = 0; h < 3; ++h) {
+          // 32 keys: exponentials, row-sum contribution, packed bf16 probabilities to tensor memory
+          auto exp_chunk = [&](int h, auto masked_tag) {
+            constexpr bool masked = decltype(masked_tag)::value;
             uint32_t pk[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
               float p0 = ex2_approx(fmaf(__uint_as_float(sv[32 * h + 2 * i]), scale, -m_ref));
               float p1 = ex2_approx(fmaf(__uint_as_float(sv[32 * h + 2 * i + 1]), scale, -m_ref));
-              if (kv_valid != kTK) {
+              if (masked) {
                 if (32 * h + 2 * i >= kv_valid) p0 = 0.f;
                 if (32 * h + 2 * i + 1 >= kv_valid) p1 = 0.f;
               }
@@ -402,6 +405,17 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
               pk[i] = *reinterpret_cast<uint32_t*>(&v);
             }
             tmem_st_32x16(ta_p + 16 * h, pk);
+          };
+          if (kv_valid == kTK) {
+            exp_chunk(0, std::false_type{});
+            exp_chunk(1, std::false_type{});
+            exp_chunk(2, std::false_type{});
+          } else {
+            // ragged last step of a sequence: only the 32-key chunks that hold a valid key (the
+            // P V product reads no probability column beyond them)
+            exp_chunk(0, std::true_type{});
+            if (kv_valid > 32) exp_chunk(1, std::true_type{});
+            if (kv_valid > 64) exp_chunk(2, std::true_type{});
           }
           l_run += rs + rs1;
           tmem_st_wait();
