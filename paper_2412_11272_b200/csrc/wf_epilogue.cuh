@@ -11,20 +11,23 @@ __device__ __forceinline__ float gelu_erf(float u) {
 }
 
 // GELU for bf16 outputs: x * sigmoid(p(x)) with the odd polynomial
-// p(x) = x (1.5950158 + 0.0740113 x^2 - 0.00070304 x^4) fitted to logit(Phi(x)); the argument of p
-// is clamped to [-8, 8] (beyond, sigmoid is 0 or 1 to 1e-12).  Max absolute deviation from the
-// erf form: 2.6e-5 over the real line, two orders of magnitude under bf16 rounding of the result.
+// p(x) = x (1.5950158 + 0.0740113 x^2 - 0.00070304 x^4) fitted to logit(Phi(x)) (max absolute
+// deviation of x * sigmoid(p(x)) from the erf form: 2.6e-5 over the real line), evaluated as
+// 0.5 x (1 + tanh(p(x) / 2)) with the hardware tanh: one special-function instruction per element
+// instead of an exponential and a reciprocal.  tanh.approx is good to 2^-11 relative, which adds
+// at most 2.5e-4 |x| to the result: an eighth of the bf16 rounding step of large outputs, and
+// below 8e-4 in absolute terms on the negative tail where the result itself is under 0.17.
 __device__ __forceinline__ float gelu_sigmoid_poly(float x) {
-  constexpr float kL2e = 1.4426950408889634f;
-  constexpr float c0 = -1.5950157568597356f * kL2e, c1 = -0.07401130190182707f * kL2e,
-                  c2 = 0.0007030350661891551f * kL2e;
-  float xc = fminf(fmaxf(x, -8.0f), 8.0f);
-  float x2 = xc * xc;
+  constexpr float c0 = 0.5f * 1.5950157568597356f, c1 = 0.5f * 0.07401130190182707f,
+                  c2 = -0.5f * 0.0007030350661891551f;
+  const float xc = fminf(fmaxf(x, -8.0f), 8.0f);  // keeps the quartic from turning p over for |x| > 8.6
+  const float x2 = xc * xc;
   float t = fmaf(x2, c2, c1);
   t = fmaf(x2, t, c0);
-  float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(xc * t));
-  return __fdividef(x, 1.0f + e);
+  float th;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(xc * t));
+  const float hx = 0.5f * x;
+  return fmaf(hx, th, hx);
 }
 
 __device__ __forceinline__ void store_elem(float* p, float v) { *p = v; }

@@ -194,6 +194,25 @@ def test_tcgen05_gemm_matches_fp64(M, N, K, mode):
     enc.close()
 
 
+def test_gelu_epilogue_pointwise():
+    """The GELU of the bf16 GEMM epilogue on a grid of arguments (fed through a one-hot GEMM so that
+    the accumulator is the argument itself) against the oracle's erf form: within bf16 rounding of
+    the result plus 1e-3 over [-12, 12], the negative tail included."""
+    shape = _small("bf16", n_layer=0)
+    enc = make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000)
+    x = I.round_to_bf16(np.concatenate([np.linspace(-12.0, 12.0, 4001), np.linspace(-1.0, 1.0, 2001)]).astype(np.float32))
+    A = np.zeros((len(x), 8), np.float32)
+    A[:, 0] = x
+    Wm = np.zeros((8, 8), np.float32)
+    Wm[:, 0] = 1.0
+    out = to_np(enc.wf_gemm_bf16(_dev(A, torch.bfloat16), _dev(Wm, torch.bfloat16), _dev(np.zeros(8, np.float32)), 1))
+    enc.wf_check()
+    ref = O.gelu(x.astype(np.float64))
+    err = np.abs(out[:, 3] - ref)
+    assert np.all(err <= 2.0 ** -8 * np.abs(ref) + 1e-3), float(np.max(err - 2.0 ** -8 * np.abs(ref)))
+    enc.close()
+
+
 @pytest.mark.parametrize("mode", [0, 2])
 def test_tcgen05_gemm_ragged_last_tile_repeated(mode):
     """M leaves whole 32-row groups of the last tile outside the matrix and N leaves 32-column
