@@ -20,6 +20,8 @@
  *   - Errors are return codes; nothing aborts.  After a non-zero return the outputs are
  *     undefined.  wf_last_error gives a human-readable message for the last failure on a
  *     handle.  A handle is not thread-safe; distinct handles are independent.
+ *   - Calls on one handle share its workspace: enqueue them on one stream, or order the streams
+ *     yourself so that two calls never run on the GPU at the same time.
  *   - Row counts: a buffer of L samples has T = floor(L/160) frames (L >= 401 required);
  *     with the hush segment of H frames it has T' = T + H rows and n = ceil(T'/2) tokens.
  */
