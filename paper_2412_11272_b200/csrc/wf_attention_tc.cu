@@ -41,7 +41,12 @@ namespace {
 
 constexpr int kTQ = 128;          // query rows per tile
 constexpr int kTK = 96;           // keys per step
-constexpr int kKvStages = 6;
+constexpr int kKvStages = 4;
+// When the two tiles of an item belong to different heads their stages alternate, tile t owning
+// every second stage; with an even count each tile's stages are its own, so neither tile ever
+// waits for the other (an odd count made them share stages and deadlock; three was tried).
+// Same-pod A/B: four stages are 0.3-1.3 % faster than six, eight are 2-3 % slower.
+static_assert(kKvStages >= 4 && kKvStages % 2 == 0, "K/V ring: even, at least four stages");
 constexpr int kQBytes = kTQ * 64 * 2;      // 16 KB
 constexpr int kKvBytes = kTK * 64 * 2;     // 12 KB
 constexpr int kAttnThreads = 352;
