@@ -13,7 +13,9 @@
 //                    are taken relative to a reference maximum that is only raised (and the
 //                    accumulator rescaled, read-modify-write in tensor memory) when the true
 //                    maximum exceeds it by more than 2^8 -- the final O / l does not depend on
-//                    that choice.  In steady state the softmax never waits for the tensor pipe.
+//                    that choice.  After an item's first step the row maximum is not even
+//                    computed unless the step's sum of probabilities shows that it is needed.
+//                    In steady state the softmax never waits for the tensor pipe.
 //   warp 8           one lane issues the TMA loads: Q tiles once per item, K and V tiles of 96
 //                    keys through two rings of kKvStages stages.
 //   warps 9, 10      MMA issue for query tile 0 / 1 (warp 9 also owns the tensor-memory
@@ -322,6 +324,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
 
     const uint32_t ta_o = ta_s + 192;
     constexpr float kRaise = 8.0f;  // the reference maximum is raised when exceeded by 2^8
+    constexpr float kRaiseSum = 256.0f;  // a probability above 2^kRaise makes the step's sum exceed this
     auto wait_warp = [&](uint32_t bar, uint32_t parity) -> bool {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
     };
@@ -348,46 +351,27 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
         tc_fence_before();
         mbar_arrive(s_free(t));  // the scores are in registers: the next S may overwrite them
         if (active) {
-          float mx = -INFINITY;
-          if (kv_valid == kTK) {
-            // four independent chains: a single running maximum would serialise 48 dependent ops
-            float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+          auto row_max = [&]() -> float {
+            float mx = -INFINITY;
+            if (kv_valid == kTK) {
+              // four independent chains: a single running maximum would serialise 48 dependent ops
+              float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < kTK; i += 8) {
-              m0 = fmaxf(m0, fmaxf(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])));
-              m1 = fmaxf(m1, fmaxf(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])));
-              m2 = fmaxf(m2, fmaxf(__uint_as_float(sv[i + 4]), __uint_as_float(sv[i + 5])));
-              m3 = fmaxf(m3, fmaxf(__uint_as_float(sv[i + 6]), __uint_as_float(sv[i + 7])));
-            }
-            mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-          } else {
-#pragma unroll
-            for (int i = 0; i < kTK; ++i)
-              if (i < kv_valid) mx = fmaxf(mx, __uint_as_float(sv[i]));
-          }
-          const float m_tile = mx * scale;  // finite: the first key of a step is always valid
-          if (j == 0) {
-            m_ref = m_tile;
-          } else {
-            const bool raise = m_tile > m_ref + kRaise;
-            if (__any_sync(0xffffffffu, raise)) {
-              // rescale this warp's accumulator rows; needs the previous P V to have landed
-              if (!wait_warp(o_full(t, (g - 1) & 1u), ((g - 1) >> 1) & 1u)) { ok = false; break; }
-              tc_fence_after();
-              const float corr = raise ? ex2_approx(m_ref - m_tile) : 1.0f;
-              if (raise) { m_ref = m_tile; l_run *= corr; }
-#pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                uint32_t a[16];
-                tmem_ld_32x16(ta_o + 16 * c, a);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 16; ++i) a[i] = __float_as_uint(__uint_as_float(a[i]) * corr);
-                tmem_st_32x16(ta_o + 16 * c, a);
+              for (int i = 0; i < kTK; i += 8) {
+                m0 = fmaxf(m0, fmaxf(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])));
+                m1 = fmaxf(m1, fmaxf(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])));
+                m2 = fmaxf(m2, fmaxf(__uint_as_float(sv[i + 4]), __uint_as_float(sv[i + 5])));
+                m3 = fmaxf(m3, fmaxf(__uint_as_float(sv[i + 6]), __uint_as_float(sv[i + 7])));
               }
-              tmem_st_wait();
+              mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+            } else {
+#pragma unroll
+              for (int i = 0; i < kTK; ++i)
+                if (i < kv_valid) mx = fmaxf(mx, __uint_as_float(sv[i]));
             }
-          }
+            return mx * scale;  // finite: the first key of a step is always valid
+          };
+          if (j == 0) m_ref = row_max();
           // The probability buffer of this step was last read by the P V of two steps ago.  That
           // product was issued, by the same thread, before the S of this step, and the commit
           // behind S tracks every earlier MMA of that thread: having seen s_full, it has landed.
@@ -411,16 +395,48 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
             }
             tmem_st_32x16(ta_p + 16 * h, pk);
           };
-          if (kv_valid == kTK) {
-            exp_chunk(0, std::false_type{});
-            exp_chunk(1, std::false_type{});
-            exp_chunk(2, std::false_type{});
-          } else {
-            // ragged last step of a sequence: only the 32-key chunks that hold a valid key (the
-            // P V product reads no probability column beyond them)
-            exp_chunk(0, std::true_type{});
-            if (kv_valid > 32) exp_chunk(1, std::true_type{});
-            if (kv_valid > 64) exp_chunk(2, std::true_type{});
+          auto exp_step = [&]() {
+            rs = 0.f;
+            rs1 = 0.f;
+            if (kv_valid == kTK) {
+              exp_chunk(0, std::false_type{});
+              exp_chunk(1, std::false_type{});
+              exp_chunk(2, std::false_type{});
+            } else {
+              // ragged last step of a sequence: only the 32-key chunks that hold a valid key (the
+              // P V product reads no probability column beyond them)
+              exp_chunk(0, std::true_type{});
+              if (kv_valid > 32) exp_chunk(1, std::true_type{});
+              if (kv_valid > 64) exp_chunk(2, std::true_type{});
+            }
+          };
+          // After the first step the probabilities are taken against the reference maximum as it
+          // stands, without looking for the step's own maximum first.  A score more than 2^8 above
+          // the reference shows in the step's sum of probabilities (> 2^8, while a step whose
+          // maximum stays below the reference sums to at most 96): only then is the maximum taken,
+          // the reference raised, the accumulator rescaled and the step's probabilities redone.
+          exp_step();
+          if (j > 0 && __any_sync(0xffffffffu, !(rs + rs1 <= kRaiseSum))) {
+            const float m_tile = row_max();
+            const bool raise = m_tile > m_ref + kRaise;
+            if (__any_sync(0xffffffffu, raise)) {
+              // rescale this warp's accumulator rows; needs the previous P V to have landed
+              if (!wait_warp(o_full(t, (g - 1) & 1u), ((g - 1) >> 1) & 1u)) { ok = false; break; }
+              tc_fence_after();
+              const float corr = raise ? ex2_approx(m_ref - m_tile) : 1.0f;
+              if (raise) { m_ref = m_tile; l_run *= corr; }
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                uint32_t a[16];
+                tmem_ld_32x16(ta_o + 16 * c, a);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) a[i] = __float_as_uint(__uint_as_float(a[i]) * corr);
+                tmem_st_32x16(ta_o + 16 * c, a);
+              }
+              tmem_st_wait();
+              exp_step();  // lanes that did not raise reproduce what they had
+            }
           }
           l_run += rs + rs1;
           tmem_st_wait();
