@@ -376,28 +376,36 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
           // product was issued, by the same thread, before the S of this step, and the commit
           // behind S tracks every earlier MMA of that thread: having seen s_full, it has landed.
           float rs = 0.f, rs1 = 0.f;
+          uint64_t acc2 = 0, acc2b = 0;  // two-wide running sums of the step's probabilities
           const uint32_t ta_p = ta_s + 96 + 48 * (g & 1u);
+          const uint64_t scale2 = pack_f32x2(scale, scale);
+          uint64_t nref2 = 0;  // (-m_ref, -m_ref), set at the start of exp_step
           // 32 keys: exponentials, row-sum contribution, packed bf16 probabilities to tensor memory
+          // (the scaling and the sums go through two-wide float32 instructions: the loop is bound by
+          // instruction issue next to the special-function unit)
           auto exp_chunk = [&](int h, auto masked_tag) {
             constexpr bool masked = decltype(masked_tag)::value;
             uint32_t pk[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              float p0 = ex2_approx(fmaf(__uint_as_float(sv[32 * h + 2 * i]), scale, -m_ref));
-              float p1 = ex2_approx(fmaf(__uint_as_float(sv[32 * h + 2 * i + 1]), scale, -m_ref));
+              float a0, a1;
+              unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[32 * h + 2 * i]), __uint_as_float(sv[32 * h + 2 * i + 1])),
+                                     scale2, nref2), a0, a1);
+              float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
               if (masked) {
                 if (32 * h + 2 * i >= kv_valid) p0 = 0.f;
                 if (32 * h + 2 * i + 1 >= kv_valid) p1 = 0.f;
               }
-              if (i & 1) rs1 += p0 + p1; else rs += p0 + p1;
+              if (i & 1) acc2b = add_f32x2(acc2b, pack_f32x2(p0, p1)); else acc2 = add_f32x2(acc2, pack_f32x2(p0, p1));
               __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
               pk[i] = *reinterpret_cast<uint32_t*>(&v);
             }
             tmem_st_32x16(ta_p + 16 * h, pk);
           };
           auto exp_step = [&]() {
-            rs = 0.f;
-            rs1 = 0.f;
+            acc2 = 0;
+            acc2b = 0;
+            nref2 = pack_f32x2(-m_ref, -m_ref);
             if (kv_valid == kTK) {
               exp_chunk(0, std::false_type{});
               exp_chunk(1, std::false_type{});
@@ -409,6 +417,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
               if (kv_valid > 32) exp_chunk(1, std::true_type{});
               if (kv_valid > 64) exp_chunk(2, std::true_type{});
             }
+            float s0, s1, s2, s3;
+            unpack_f32x2(acc2, s0, s1);
+            unpack_f32x2(acc2b, s2, s3);
+            rs = s0 + s1;
+            rs1 = s2 + s3;
           };
           // After the first step the probabilities are taken against the reference maximum as it
           // stands, without looking for the step's own maximum first.  A score more than 2^8 above
