@@ -55,7 +55,7 @@ __device__ __forceinline__ void bias_act32(const EpiParams& ep, int col0, int N,
   }
   if (EPI == kEpiBiasGelu || EPI == kEpiConv1 || EPI == kEpiConv2) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = gelu_sigmoid_poly(v[i]);
+    for (int i = 0; i < 32; i += 2) gelu_sigmoid_poly2(v[i], v[i + 1]);
   }
 }
 
