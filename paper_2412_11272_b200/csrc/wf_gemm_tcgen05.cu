@@ -48,10 +48,10 @@ __device__ __forceinline__ void bias_act32(const EpiParams& ep, int col0, int N,
   for (int g = 0; g < 8; ++g) {
     int col = col0 + 4 * g;
     float4 b = (col < N && with_bias) ? __ldg(reinterpret_cast<const float4*>(ep.bias + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    v[4 * g + 0] = __uint_as_float(acc[4 * g + 0]) + b.x;
-    v[4 * g + 1] = __uint_as_float(acc[4 * g + 1]) + b.y;
-    v[4 * g + 2] = __uint_as_float(acc[4 * g + 2]) + b.z;
-    v[4 * g + 3] = __uint_as_float(acc[4 * g + 3]) + b.w;
+    unpack_f32x2(add_f32x2(pack_f32x2(__uint_as_float(acc[4 * g + 0]), __uint_as_float(acc[4 * g + 1])),
+                           pack_f32x2(b.x, b.y)), v[4 * g + 0], v[4 * g + 1]);
+    unpack_f32x2(add_f32x2(pack_f32x2(__uint_as_float(acc[4 * g + 2]), __uint_as_float(acc[4 * g + 3])),
+                           pack_f32x2(b.z, b.w)), v[4 * g + 2], v[4 * g + 3]);
   }
   if (EPI == kEpiBiasGelu || EPI == kEpiConv1 || EPI == kEpiConv2) {
 #pragma unroll
