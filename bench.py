@@ -35,7 +35,7 @@ N_STREAMS = 64
 ROUNDS = list(range(1, 16))
 # DRAM bytes per token of the four block GEMMs (QKV, out-proj, FC1, FC2), from the ncu capture
 # summarised in profiles/gemm_bf16_pair_M16384.md (M = 16384; traffic grows in proportion to M)
-GEMM_DRAM_BYTES_PER_TOKEN = (7714.0, 9448.0, 10479.0, 21101.0)
+GEMM_DRAM_BYTES_PER_TOKEN = (7758.0, 9448.0, 10565.0, 20960.0)
 SAMPLE_SECONDS = 15         # the CPU oracle is timed on stream 0's full 15 s window (775 tokens)
 
 
