@@ -43,6 +43,7 @@ namespace {
 
 constexpr int kTQ = 128;          // query rows per tile
 constexpr int kTK = 96;           // keys per step
+constexpr int kPolyEvery = 4;  // every 4th pair of exponentials is evaluated on the FMA pipe (0: none)
 constexpr int kKvStages = 4;
 // When the two tiles of an item belong to different heads their stages alternate, tile t owning
 // every second stage; with an even count each tile's stages are its own, so neither tile ever
@@ -391,7 +392,29 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
               float a0, a1;
               unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[32 * h + 2 * i]), __uint_as_float(sv[32 * h + 2 * i + 1])),
                                      scale2, nref2), a0, a1);
-              float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
+              float p0, p1;
+              if (kPolyEvery > 0 && (i % kPolyEvery) == kPolyEvery - 1) {
+                // 2^a on the FMA pipe for every kPolyEvery-th pair (the special-function unit is the
+                // loop's limit): a = j + f with j the nearest integer (magic-number rounding) and
+                // |f| <= 0.5, 2^f by a cubic (relative error 8e-5, far below bf16 rounding of the
+                // probability), j added to the exponent bits.  a >= -120 keeps the exponent in range.
+                const uint64_t ax = pack_f32x2(fmaxf(a0, -120.0f), fmaxf(a1, -120.0f));
+                const uint64_t tt = add_f32x2(ax, pack_f32x2(12582912.0f, 12582912.0f));
+                const uint64_t jj = add_f32x2(tt, pack_f32x2(-12582912.0f, -12582912.0f));
+                const uint64_t ff = fma_f32x2(jj, pack_f32x2(-1.0f, -1.0f), ax);
+                uint64_t pp = fma_f32x2(ff, pack_f32x2(0.05508868396282196f, 0.05508868396282196f),
+                                        pack_f32x2(0.24260404706001282f, 0.24260404706001282f));
+                pp = fma_f32x2(ff, pp, pack_f32x2(0.6932762265205383f, 0.6932762265205383f));
+                pp = fma_f32x2(ff, pp, pack_f32x2(0.9999289512634277f, 0.9999289512634277f));
+                float t0, t1, q0, q1;
+                unpack_f32x2(tt, t0, t1);
+                unpack_f32x2(pp, q0, q1);
+                p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+                p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+              } else {
+                p0 = ex2_approx(a0);
+                p1 = ex2_approx(a1);
+              }
               if (masked) {
                 if (32 * h + 2 * i >= kv_valid) p0 = 0.f;
                 if (32 * h + 2 * i + 1 >= kv_valid) p1 = 0.f;
