@@ -506,8 +506,9 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
   WF_TRY(dev_alloc<float>(e, &e->pe, (size_t)c.n_ctx * d));
   launch_build_tables(e->dft_basis, e->pe, c.n_ctx, d, s);
   if (!w->mel_fb) return fail(e, WF_ERR_INVALID_ARG, "mel_fb is NULL");
-  WF_TRY(dev_alloc<float>(e, &e->mel_fb_t, (size_t)kBins * c.n_mel));
+  WF_TRY(dev_alloc<float>(e, &e->mel_fb_t, (size_t)kBins * c.n_mel + 2 * c.n_mel));
   launch_transpose_f32(w->mel_fb, e->mel_fb_t, c.n_mel, kBins, s);
+  launch_mel_bin_ranges(e->mel_fb_t, c.n_mel, s);
   // conv stem
   WF_TRY(dev_alloc_bytes(e, &e->conv1_w, (size_t)d * 3 * e->mel_ld * e->esz, true));
   WF_TRY(dev_alloc_bytes(e, &e->conv2_w, (size_t)d * 3 * d * e->esz, true));

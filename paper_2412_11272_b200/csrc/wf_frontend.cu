@@ -106,6 +106,7 @@ __global__ void __launch_bounds__(256) frontend_kernel(
   const float* x = audio + s0;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+#pragma unroll 5
   for (int idx = tid; idx < kFeFrames * kFold; idx += 256) {
     int f = idx / kFold, n = idx % kFold + 1;
     int t = t0 + f;
@@ -207,18 +208,25 @@ __global__ void __launch_bounds__(256) frontend_kernel(
 #pragma unroll
     for (int j = 0; j < 4; ++j) mel[f][j] = 0.f;
   const float* pr = p_s + warp * 8 * kPStride;
-  for (int k = 0; k < kBins; ++k) {
-    float w[4];
+  // Filterbanks are sparse (a channel is fed by a short run of neighbouring bins): the first and
+  // last bin with a non-zero weight of every channel sit behind the transposed filterbank, and a
+  // lane walks only its channels' runs, in ascending bin order as the full product would (the
+  // skipped products would have added exact zeros; lanes past the end of their run add one).
+  const int2* bin_range = reinterpret_cast<const int2*>(fbt + kBins * n_mel);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      int m = lane + 32 * j;
-      w[j] = m < n_mel ? __ldg(fbt + k * n_mel + m) : 0.f;
-    }
+  for (int j = 0; j < 4; ++j) {
+    const int m = lane + 32 * j;
+    const int2 rg = m < n_mel ? __ldg(bin_range + m) : make_int2(0, 0);
+    int len = rg.y - rg.x;
 #pragma unroll
-    for (int f = 0; f < 8; ++f) {
-      float p = pr[f * kPStride + k];
+    for (int o = 16; o > 0; o >>= 1) len = max(len, __shfl_xor_sync(0xffffffffu, len, o));
+    for (int kk = 0; kk < len; ++kk) {
+      const int k = rg.x + kk;
+      const bool in_run = k < rg.y;
+      const int kc = in_run ? k : 0;
+      const float wj = in_run ? __ldg(fbt + kc * n_mel + m) : 0.f;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) mel[f][j] = fmaf(p, w[j], mel[f][j]);
+      for (int f = 0; f < 8; ++f) mel[f][j] = fmaf(pr[f * kPStride + kc], wj, mel[f][j]);
     }
   }
   float mx = -INFINITY;
@@ -411,6 +419,25 @@ void launch_build_maps(const int* meta, MetaLayout ml, int B, int max_rows, int 
   if (B <= 0 || max_rows <= 0) return;
   dim3 grid((max_rows + 255) / 256, B);
   build_maps_kernel<<<grid, 256, 0, s>>>(meta, ml, hush_frames, row_valid, row_dst);
+}
+
+// Behind the transposed filterbank [201][n_mel]: per channel the half-open run of bins [first, last + 1)
+// that holds all its non-zero weights (0, 0 for an all-zero channel).
+__global__ void mel_bin_range_kernel(float* fbt, int n_mel) {
+  const int m = blockIdx.x * blockDim.x + threadIdx.x;
+  if (m >= n_mel) return;
+  int lo = 0, hi = 0;
+  bool any = false;
+  for (int k = 0; k < kBins; ++k)
+    if (fbt[k * n_mel + m] != 0.f) {
+      if (!any) lo = k;
+      any = true;
+      hi = k + 1;
+    }
+  reinterpret_cast<int2*>(fbt + kBins * n_mel)[m] = make_int2(lo, hi);
+}
+void launch_mel_bin_ranges(float* mel_fb_t, int n_mel, cudaStream_t s) {
+  mel_bin_range_kernel<<<1, 128, 0, s>>>(mel_fb_t, n_mel);
 }
 
 }  // namespace wf

@@ -93,6 +93,9 @@ void launch_build_tables(float* dft_basis /*[2][kFold][kBasisCols]*/, float* pe,
                          cudaStream_t s);
 
 // ---- front end (wf_frontend.cu)
+// mel_fb_t holds the transposed filterbank [201][n_mel] followed by n_mel int2 (launch_mel_bin_ranges):
+// per channel, the run of bins [first, last + 1) that holds its non-zero weights.
+void launch_mel_bin_ranges(float* mel_fb_t, int n_mel, cudaStream_t s);
 void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, int n_tiles,
                      const float* dft_basis, const float* mel_fb_t /*[201][n_mel]*/, int n_mel,
                      float* logmel /*[sum T, n_mel]*/, int* seq_max /*[B] ordered ints*/,
