@@ -72,6 +72,7 @@ void launch_fill_seq_max(int* seq_max, int B, cudaStream_t s) {
 // the mel projection, log10 and the per-buffer running maximum.
 constexpr int kPStride = 204;
 constexpr int kBasisChunk = 8;  // folded-DFT rows per staged chunk (a multiple of 4 that divides 200)
+constexpr int kFeSpan = kHop * (kFeFrames - 1) + 399;  // samples one tile of frames touches
 constexpr int kFeSmemFloats = kFeFrames * kPStride > 2 * kFeFrames * kFold ? kFeFrames * kPStride : 2 * kFeFrames * kFold;
 
 __global__ void __launch_bounds__(256) frontend_kernel(
@@ -106,24 +107,32 @@ __global__ void __launch_bounds__(256) frontend_kernel(
   const float* x = audio + s0;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-#pragma unroll 5
-  for (int idx = tid; idx < kFeFrames * kFold; idx += 256) {
-    int f = idx / kFold, n = idx % kFold + 1;
-    int t = t0 + f;
-    float e = 0.f, o = 0.f;
-    if (t < T) {
-      int c = kHop * t;
-      int ia = c - 200 + n, ib = c + 200 - n;
-      if (ia < 0) ia = -ia;
-      if (ia >= L) ia = 2 * (L - 1) - ia;
-      if (ib < 0) ib = -ib;
-      if (ib >= L) ib = 2 * (L - 1) - ib;
-      float a = ia < L_audio ? x[ia] : tail[ia - L_audio];
-      if (n == kFold) { e = a; }
-      else { float b = ib < L_audio ? x[ib] : tail[ib - L_audio]; e = a + b; o = a - b; }
+  // The tile's samples (with the reflected ends and the raw-audio hush word resolved) go to shared
+  // memory once, coalesced; the fold then reads every sample twice from there instead of from
+  // global memory.
+  {
+    float* span = smem + kFeSmemFloats + 2 * 2 * kBasisChunk * kBasisCols;
+    const int p0 = kHop * t0 - 199;  // span[i] is sample p0 + i
+#pragma unroll 4
+    for (int i = tid; i < kFeSpan; i += 256) {
+      int p = p0 + i;
+      if (p < 0) p = -p;
+      if (p >= L) p = 2 * (L - 1) - p;
+      p = min(max(p, 0), L - 1);  // only for frames past the end of the buffer, which are not used
+      span[i] = p < L_audio ? x[p] : tail[p - L_audio];
     }
-    e_s[idx] = e;
-    o_s[idx] = o;
+    __syncthreads();
+    for (int idx = tid; idx < kFeFrames * kFold; idx += 256) {
+      const int f = idx / kFold, n = idx % kFold + 1;
+      float e = 0.f, o = 0.f;
+      if (t0 + f < T) {
+        const float a = span[kHop * f - 1 + n];          // sample c - 200 + n, c = 160 (t0 + f)
+        if (n == kFold) { e = a; }
+        else { const float b = span[kHop * f + 399 - n]; e = a + b; o = a - b; }  // sample c + 200 - n
+      }
+      e_s[idx] = e;
+      o_s[idx] = o;
+    }
   }
   __syncthreads();
 
@@ -254,7 +263,7 @@ __global__ void __launch_bounds__(256) frontend_kernel(
 void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, int n_tiles,
                      const float* dft_basis, const float* mel_fb_t, int n_mel, float* logmel,
                      int* seq_max, const float* tail, int tail_len, cudaStream_t s) {
-  const int smem = (kFeSmemFloats + 2 * 2 * kBasisChunk * kBasisCols) * (int)sizeof(float);  // 102,400 + 28,672 B
+  const int smem = (kFeSmemFloats + 2 * 2 * kBasisChunk * kBasisCols + kFeSpan + 1) * (int)sizeof(float);  // 172,992 B
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(frontend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
