@@ -11,14 +11,18 @@ reference for the current decoding session.
 * fallback -- if the alignment search finds nothing, or a comparable token differs from
   reference[i], the beam returns to its full size.
 
-Readings where the text leaves a choice (also listed in the design doc):
+Readings where the text leaves a choice:
   R1  the alignment search uses the first top-1 token that is comparable (a leading timestamp or
       other special token is skipped like any other special token);
   R2  the aligned token counts as matched: after a hit at position i the next comparison is with
       reference[i + 1];
   R3  once the reference is exhausted a comparable token has nothing to match and triggers the
       fallback;
-  R4  the fallback lasts until the end of the decoding session.
+  R4  the fallback lasts until the end of the decoding session;
+  R5  punctuation, timestamp and special tokens are skipped on the reference side as well: the
+      previous round's transcript carries them too, and a word must not be compared with a comma
+      the model happened to emit last time.  The reference index rests right behind the last
+      matched token; before a comparison it passes over special reference entries.
 This module is independent of the library: plain Python, no shared code.
 """
 from __future__ import annotations
@@ -46,8 +50,11 @@ class BeamPruner:
                     return 1
             self.fallen_back = True
             return self.full
-        if self.i < len(self.ref) and self.ref[self.i] == top1:
-            self.i += 1
+        j = self.i
+        while j < len(self.ref) and self.ref[j] in self.special:     # R5
+            j += 1
+        if j < len(self.ref) and self.ref[j] == top1:
+            self.i = j + 1
             return 1
         self.fallen_back = True                               # mismatch, or reference exhausted (R3)
         return self.full

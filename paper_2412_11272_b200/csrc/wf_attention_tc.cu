@@ -397,8 +397,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) attention_tc_kernel(
                 // 2^a on the FMA pipe for every kPolyEvery-th pair (the special-function unit is the
                 // loop's limit): a = j + f with j the nearest integer (magic-number rounding) and
                 // |f| <= 0.5, 2^f by a cubic (relative error 8e-5, far below bf16 rounding of the
-                // probability), j added to the exponent bits.  a >= -120 keeps the exponent in range.
-                const uint64_t ax = pack_f32x2(fmaxf(a0, -120.0f), fmaxf(a1, -120.0f));
+                // probability), j added to the exponent bits.  -120 <= a <= 127 keeps the exponent in
+                // range: a score far above the reference then gives 2^127 (not a wrapped exponent), which
+                // drives the step's sum over the raise threshold exactly as the ex2 lanes' +inf does.
+                const uint64_t ax = pack_f32x2(fminf(fmaxf(a0, -120.0f), 127.0f), fminf(fmaxf(a1, -120.0f), 127.0f));
                 const uint64_t tt = add_f32x2(ax, pack_f32x2(12582912.0f, 12582912.0f));
                 const uint64_t jj = add_f32x2(tt, pack_f32x2(-12582912.0f, -12582912.0f));
                 const uint64_t ff = fma_f32x2(jj, pack_f32x2(-1.0f, -1.0f), ax);

@@ -4,7 +4,8 @@
 // Decoding starts with beam size 1.  The first comparable top-1 token is searched through the
 // reference (search-based alignment); afterwards each comparable top-1 token must equal the next
 // reference token to keep the beam at 1; punctuation, timestamp and other special tokens are
-// never compared; a failed search or a mismatch restores the full beam for the rest of the session.
+// never compared -- neither as the top-1 token nor as reference entries, which the reference
+// index passes over; a failed search or a mismatch restores the full beam for the rest of the session.
 #include <new>
 #include <vector>
 
@@ -59,12 +60,19 @@ int wf_beam_pruner_step(wf_beam_pruner* p, int top1_token) {
         break;
       }
     }
-  } else if (p->index < (long)p->ref.size() && p->ref[p->index] == top1_token) {
-    ++p->index;
-    next = 1;
   } else {
-    p->fallen_back = true;
-    next = p->full_beam;
+    // the comparison target is the next reference entry that is not itself punctuation, a
+    // timestamp or another special token (the previous transcript carries those as well)
+    long at = p->index;
+    const long n_ref = (long)p->ref.size();
+    while (at < n_ref && p->special[p->ref[at]]) ++at;
+    if (at < n_ref && p->ref[at] == top1_token) {
+      p->index = at + 1;
+      next = 1;
+    } else {
+      p->fallen_back = true;
+      next = p->full_beam;
+    }
   }
   ++p->rounds;
   if (next == 1) ++p->rounds_at_one;

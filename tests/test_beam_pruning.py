@@ -48,6 +48,22 @@ def test_first_match_is_taken_when_the_token_repeats():
     assert p.step(60) == 1 and p.step(50) == 1 and p.step(61) == 1 and p.i == 4
 
 
+def test_special_tokens_inside_the_reference_are_passed_over():
+    # the previous transcript "50 , 51 <ts> 52" against "50 , 51 52": the comma and the timestamp of
+    # the reference are no comparison targets, so 51 meets 51 and 52 meets 52
+    beams, idx, fb = BO.run_session([50, 7, 51, 3, 52], SPECIAL, [50, 7, 51, 52])
+    assert beams == [1, 1, 1, 1] and idx == 5 and not fb
+    # punctuation on one side only, either side
+    beams, idx, fb = BO.run_session([50, 7, 51, 52], SPECIAL, [50, 51, 9, 52])
+    assert beams == [1, 1, 1, 1] and idx == 4 and not fb
+    # a real mismatch behind a reference comma still falls back, and the index stays behind the last match
+    beams, idx, fb = BO.run_session([50, 7, 51], SPECIAL, [50, 60, 51])
+    assert beams == [1, 1, 5] and fb and idx == 1
+    # a reference that ends in punctuation is exhausted for a new word
+    beams, idx, fb = BO.run_session([50, 7], SPECIAL, [50, 70])
+    assert beams == [1, 1] and fb and idx == 1
+
+
 # ----- the library against the oracle ----------------------------------------------------------------
 
 def _stream(seed, n):
@@ -62,6 +78,9 @@ def test_library_matches_oracle_on_synthetic_sessions():
     for seed in range(200):
         prev = _stream(seed, 40)
         u = I.uniform01(seed, 78, 200)
+        if seed % 2:                                        # previous transcripts carry punctuation / timestamps too
+            v = I.uniform01(seed, 79, 80)
+            prev = [t for k, t in enumerate(prev) for t in ([int(v[40 + k] * 20)] if v[k] < 0.2 else []) + [t]]
         cut = int(u[0] * 10)                                # audio trimmed at the front
         cur = prev[cut:] + _stream(seed + 1000, 8)          # and new audio appended at the end
         out = []

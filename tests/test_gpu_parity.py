@@ -326,6 +326,30 @@ def test_varlen_attention_matches_oracle(dtype):
         s = slice(cu[i], cu[i + 1])
         ref = O.attention(q3_64[s, :256], q3_64[s, 256:512], q3_64[s, 512:], 4)
         assert np.max(np.abs(out3[s] - ref)) < (4e-2 if dtype == "bf16" else 1e-4), (i, lens[i])   # logits up to ~60
+    # one key far above everything seen before it, sitting where the tensor-core kernel evaluates 2^a on
+    # the FMA pipe (in-step key indices 6, 7, 14, 15, ... of a 96-key step) in a step after the first:
+    # the reference maximum must be raised there too.  Every query of the sequence carries a constant
+    # in channel 0 of each head, the chosen keys a large value in the same channel.
+    q4 = qkv.copy()
+    def spike(seq, key, nats):
+        rows = slice(cu[seq], cu[seq + 1])
+        for h in range(4):
+            q4[rows, 64 * h] = 8.0
+            q4[cu[seq] + key, 256 + 64 * h] = nats
+    spike(4, 96 + 6, 150.0)                 # 200 keys: second step, FMA-pipe lane
+    spike(5, 3 * 96 + 7, 130.0)             # 1525 keys: two such keys in two different steps,
+    spike(5, 9 * 96 + 31, 280.0)            # the later one higher again
+    if dtype == "bf16":
+        q4 = I.round_to_bf16(q4)
+    out4 = to_np(enc.wf_attention(_dev(q4, tdt), cu))
+    enc.wf_check()
+    q4_64 = q4.astype(np.float64)
+    for i in (4, 5):
+        s = slice(cu[i], cu[i + 1])
+        ref = O.attention(q4_64[s, :256], q4_64[s, 256:512], q4_64[s, 512:], 4)
+        assert np.max(np.abs(out4[s] - ref)) < tol, (i, lens[i])
+    key = cu[5] + 9 * 96 + 31                # the dominant key's value row comes back for every query
+    assert np.max(np.abs(out4[cu[5]:cu[6]] - q4_64[key, 512:])) < tol
     # identical keys -> mean of values
     q2 = qkv.copy()
     q2[:, 256:512] = q2[0, 256:512]

@@ -138,6 +138,15 @@ def test_hush_append_levels():
     h_audio = I.hush_audio(9)
     xa = O.append_hush_audio(x, h_audio)
     assert len(xa) == 3200 + 8000 and O.n_tokens(O.n_frames(len(xa))) == 10 + 25
+    # x (+) h: the buffer first, the hush word behind it (Sec. 4.1.2), sample for sample
+    assert np.array_equal(xa[:3200], x.astype(np.float64)) and np.array_equal(xa[3200:], h_audio.astype(np.float64))
+    assert not np.array_equal(xa[:8000], h_audio.astype(np.float64))
+    # at the raw-audio level the junction frames mix buffer and hush samples, so the rows before the
+    # junction differ from the buffer's own log-mel rows only near it (frame t reads samples
+    # 160 t - 200 .. 160 t + 199) and through the shared maximum
+    lone, joint = O.dft_power(x), O.dft_power(xa)
+    assert np.allclose(joint[:19], lone[:19], rtol=1e-12, atol=1e-18)      # frames 0..18 end at sample 3079
+    assert not np.allclose(joint[19], lone[19], rtol=1e-3)                  # frame 19 reaches into the hush word
 
 
 # ----- encoder pieces ------------------------------------------------------------------------
@@ -288,18 +297,22 @@ def test_batch_invariance():
 
 # ----- second, independent scalar evaluation of the whole path on tiny dims ------------------
 
-def _scalar_encode(x, F, hush, W, n_layer, n_head):
+def _scalar_encode(x, F, hush, W, n_layer, n_head, hush_audio=None):
     """Pure-Python scalar evaluation in a different loop order (output-element outer loops,
-    math.fsum reductions, Python complex exponentials)."""
-    L = len(x)
+    math.fsum reductions, Python complex exponentials).  ``hush`` is the log-mel-level hush
+    segment (rows appended after the normalisation); ``hush_audio`` the raw-audio-level one:
+    its samples follow the buffer's, read through index arithmetic (no concatenated copy), and
+    the framing, the maximum and the clamp then run over the whole of x (+) h."""
+    Lx = len(x)
+    L = Lx + (len(hush_audio) if hush_audio is not None else 0)
     T = L // 160
 
-    def xs(i):                       # reflected sample
+    def xs(i):                       # reflected sample of x (+) h
         if i < 0:
             i = -i
         if i >= L:
             i = 2 * L - 2 - i
-        return float(x[i])
+        return float(x[i]) if i < Lx else float(hush_audio[i - Lx])
 
     n_mel = len(F)
     lg = [[0.0] * n_mel for _ in range(T)]
@@ -315,7 +328,9 @@ def _scalar_encode(x, F, hush, W, n_layer, n_head):
         for m in range(n_mel):
             lg[t][m] = math.log10(max(math.fsum(float(F[m][k]) * power[k] for k in range(201)), 1e-10))
     mx = max(max(r) for r in lg)
-    Z = [[(max(v, mx - 8.0) + 4.0) / 4.0 for v in r] for r in lg] + [[float(v) for v in r] for r in hush]
+    Z = [[(max(v, mx - 8.0) + 4.0) / 4.0 for v in r] for r in lg]
+    if hush is not None:
+        Z = Z + [[float(v) for v in r] for r in hush]
 
     def gelu(u):
         return 0.5 * u * (1.0 + math.erf(u / math.sqrt(2.0)))
@@ -388,6 +403,24 @@ def test_whole_path_against_scalar_evaluation(n_samples):
     ref = _scalar_encode(x, F, hush, W, 1, 2)
     assert got.shape == ref.shape == ((n_samples // 160 + 3 + 1) // 2, 8)
     assert np.max(np.abs(got - ref)) < 1e-10
+
+
+@pytest.mark.parametrize("n_samples,n_hush", [(480, 480), (640, 410)])      # T = 6 and 6 (1050 // 160): junction mid-frame
+def test_whole_path_raw_audio_hush_against_scalar_evaluation(n_samples, n_hush):
+    """The raw-audio-level variant (Sec. 4.1.2): hush samples behind the buffer's, everything
+    downstream over x (+) h.  A hush word put in front, framed separately, or left out of the
+    maximum would each move the result."""
+    shape = _tiny_shape()
+    W = {k: v.astype(np.float64) * 15 for k, v in I.encoder_weights(8, shape, bf16=False).items()}
+    F = I.mel_filterbank(4)
+    x = I.synth_audio(8, 0, n_samples)
+    h = 3.0 * I.hush_audio(8, n_hush)                   # louder than the buffer: the maximum sits in the hush part
+    got = O.encode_sequence(x, F, h, W, 1, 2, hush_level="audio")
+    ref = _scalar_encode(x, F, None, W, 1, 2, hush_audio=h)
+    assert got.shape == ref.shape == (((n_samples + n_hush) // 160 + 1) // 2, 8)
+    assert np.max(np.abs(got - ref)) < 1e-10
+    swapped = O.encode_sequence(h, F, x, W, 1, 2, hush_level="audio")
+    assert np.max(np.abs(swapped - ref)) > 1e-3
 
 
 # ----- planted mistakes: each pin set must catch a plausible slip ----------------------------
