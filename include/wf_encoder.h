@@ -51,8 +51,9 @@ typedef enum { WF_F32 = 0, WF_BF16 = 1 } wf_dtype;
 /* Model and capacity description.  d_model / n_head must be 64; d_model and d_mlp multiples
  * of 128 (d_model <= 1280); n_mel a multiple of 8, at most 128.  dtype selects the arithmetic
  * of the encoder body: WF_F32 = float32 SIMT kernels, WF_BF16 = bfloat16 tensor-core kernels
- * with float32 accumulation, float32 residual stream, bfloat16 output.  The front end is
- * float32 in both. */
+ * with float32 accumulation, a residual stream held to 16 significant bits (two bfloat16
+ * planes), each LayerNorm's gain folded into the weight that follows it (the product is
+ * rounded to bfloat16), bfloat16 output.  The front end is float32 in both. */
 typedef struct {
   int n_mel, d_model, n_layer, n_head, d_mlp;
   int n_ctx;          /* most tokens one sequence may have (positions are a closed form)   */
@@ -84,15 +85,14 @@ typedef struct {
  * the stated capacities.  Synchronises `stream` before returning.  Fails with
  * WF_ERR_UNSUPPORTED_ARCH on a device that is not compute capability 10.x.
  * (Operation: the encoder of Sec. 1.1 / Sec. 2.3; weights are caller-provided.)
- * Three process-wide tuning switches of the WF_BF16 path are read from the environment here:
+ * Two tuning switches of the WF_BF16 path are read from the environment here and kept in the
+ * handle (a later create with another environment does not change this one):
  *   WF_PDL=0               launch kernels plainly instead of with programmatic stream
  *                          serialization (on by default: a kernel's set-up overlaps the tail of
  *                          the kernel before it);
- *   WF_GEMM_SMALL_TILES=0  never use 128 x 128 single-CTA tiles for small GEMMs;
- *   WF_GEMM_TAIL_SPLIT=1   cut the last partial round of a residual GEMM's tiles along K (faster
- *                          at small M; results then vary in the last bit from run to run, which
- *                          is why it is off by default).
- * None of them changes what is computed beyond float32 rounding order. */
+ *   WF_GEMM_SMALL_TILES=0  never use 128 x 128 single-CTA tiles for small GEMMs.
+ * Neither changes what is computed.  Results are bit-reproducible from call to call: no kernel of
+ * the encoder combines partial results in an order that varies. */
 wf_status wf_encoder_create(const wf_config *cfg, const wf_weights *w, void *stream,
                             wf_encoder **out);
 
@@ -152,7 +152,8 @@ const char *wf_last_error(const wf_encoder *enc);
 
 /* Per-kernel-class timing.  When enabled, every launch inside wf_encode* is bracketed by
  * CUDA events on the caller's stream.  wf_profile_read synchronises, then writes for class c
- * (0 front end, 1 layout/maps, 2 conv stem GEMMs, 3 LayerNorm, 4 block GEMMs, 5 attention)
+ * (0 front end, 1 layout/maps, 2 conv stem GEMMs, 3 LayerNorm kernels (WF_BF16: the final one
+ * only), 4 block GEMMs, 5 attention)
  * the number of launches and their summed milliseconds since the last read, and resets. */
 #define WF_N_KERNEL_CLASSES 6
 wf_status wf_profile_enable(wf_encoder *enc, int on);
@@ -163,11 +164,37 @@ wf_status wf_profile_read(wf_encoder *enc, long *launches, double *millis);
  * wf_gemm_bf16: C = epilogue(A W^T + bias) with the tcgen05 kernel the encoder blocks use
  * (the four GEMMs of a transformer block, Sec. 1.1).  Needs a WF_BF16 encoder.
  *   A dev bf16 [M, K] row-major, W dev bf16 [N, K] row-major, bias dev float32 [N];
- *   mode 0: C bf16 [M, N] = acc + bias;  1: C bf16 = gelu(acc + bias);
- *   mode 2: C float32 [M, N] += acc + bias (residual update in place).
+ *   mode 0: C bf16 [M, N] = acc + bias;  1: C bf16 = gelu(acc + bias).
  *   K and N must be multiples of 8. */
 wf_status wf_gemm_bf16(wf_encoder *enc, const void *A, const void *W, const float *bias, void *C,
                        long M, int N, int K, int mode, void *stream);
+
+/* The three pieces with which the WF_BF16 path runs a pre-LN block (x += Wo attn(LN1 x) + bo;
+ * x += W2 gelu(W1 LN2 x + b1) + b2, the blocks of the encoder of Sec. 1.1 / Sec. 2.3) without a
+ * LayerNorm kernel: the residual stream x is stored as two bf16 planes, x = x_hi + x_lo with
+ * x_hi = bf16(x) and x_lo = bf16(x - x_hi); x_hi doubles as the A operand of the GEMM behind a
+ * LayerNorm, whose gain and shift are folded into that GEMM's weight and bias.
+ *
+ * wf_gemm_resid_bf16: (x_hi, x_lo) <- split(x_hi + x_lo + A W^T + bias), in place, each element
+ *   by one thread (bit-reproducible).  Also writes, for every row and every 128 columns, the sum
+ *   and the sum of squares of the new x:
+ *   A dev bf16 [M, K], W dev bf16 [N, K], bias dev float32 [N], x_hi / x_lo dev bf16 [M, N],
+ *   stats dev float32 [N / 128][M][2];  N a multiple of 128, K of 8.
+ * wf_ln_fold: W dev float32 [N, K], ln_g / ln_b dev float32 [K], bias dev float32 [N] or NULL ->
+ *   Wg dev bf16 [N, K] = bf16(W diag(ln_g)), colsum dev float32 [N] = row sums of Wg,
+ *   cbias dev float32 [N] = bias + W ln_b.
+ * wf_gemm_ln_bf16: C bf16 [M, N] = LayerNorm(x; ln_g, ln_b) W^T + bias (gelu of it if `gelu`),
+ *   computed as rstd (x_hi Wg^T - mean colsum) + cbias with mean and rstd (biased variance,
+ *   eps 1e-5) from `stats` [K / 128][M][2] as wf_gemm_resid_bf16 leaves them for an x of K columns.
+ *   K a multiple of 128, N of 8. */
+wf_status wf_gemm_resid_bf16(wf_encoder *enc, const void *A, const void *W, const float *bias,
+                             void *x_hi, void *x_lo, float *stats, long M, int N, int K, void *stream);
+wf_status wf_ln_fold(wf_encoder *enc, const float *W, const float *ln_g, const float *ln_b,
+                     const float *bias, void *Wg, float *colsum, float *cbias, int N, int K,
+                     void *stream);
+wf_status wf_gemm_ln_bf16(wf_encoder *enc, const void *x_hi, const float *stats, const void *Wg,
+                          const float *colsum, const float *cbias, void *C, long M, int N, int K,
+                          int gelu, void *stream);
 
 /* wf_attention: non-causal attention over packed tokens, one softmax per (sequence, head)
  * over that sequence's keys only (no padded token is computed).  qkv dev [M, 3 d_model]

@@ -83,6 +83,9 @@ def load_library() -> C.CDLL:
     lib.wf_profile_enable.argtypes = [vp, C.c_int]
     lib.wf_profile_read.argtypes = [vp, lp, C.POINTER(C.c_double)]
     lib.wf_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, C.c_long, C.c_int, C.c_int, C.c_int, vp]
+    lib.wf_gemm_resid_bf16.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.c_long, C.c_int, C.c_int, vp]
+    lib.wf_ln_fold.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, C.c_int, C.c_int, vp]
+    lib.wf_gemm_ln_bf16.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.c_long, C.c_int, C.c_int, C.c_int, vp]
     lib.wf_attention.argtypes = [vp, vp, ip, C.c_int, vp, vp]
     lib.wf_cross_kv.argtypes = [vp, vp, vp, vp, C.c_long, C.c_int, vp, vp]
     lib.wf_streams_create.argtypes = [vp, C.c_int, C.c_long, C.POINTER(vp)]
@@ -270,6 +273,38 @@ class Encoder:
         self._check(self.lib.wf_gemm_bf16(self.handle, A.data_ptr(), W.data_ptr(), bias.data_ptr(),
                                           C_out.data_ptr(), M, N, K, mode, _stream_ptr(stream)))
         return C_out
+
+    def wf_gemm_resid_bf16(self, A: torch.Tensor, W: torch.Tensor, bias: torch.Tensor, x_hi: torch.Tensor,
+                           x_lo: torch.Tensor, stream=None):
+        """(x_hi, x_lo) <- split(x_hi + x_lo + A W^T + bias) in place; returns the row statistics
+        [N / 128, M, 2] (sum and sum of squares of every 128 columns of the new x)."""
+        M, K = A.shape
+        N = W.shape[0]
+        stats = torch.empty((max(N // 128, 1), M, 2), dtype=torch.float32, device=A.device)
+        self._check(self.lib.wf_gemm_resid_bf16(self.handle, A.data_ptr(), W.data_ptr(), bias.data_ptr(), x_hi.data_ptr(),
+                                                x_lo.data_ptr(), stats.data_ptr(), M, N, K, _stream_ptr(stream)))
+        return stats
+
+    def wf_ln_fold(self, W: torch.Tensor, ln_g: torch.Tensor, ln_b: torch.Tensor, bias: torch.Tensor | None, stream=None):
+        """W float32 [N, K] -> (Wg bf16 [N, K], colsum float32 [N], cbias float32 [N])."""
+        N, K = W.shape
+        Wg = torch.empty((N, K), dtype=torch.bfloat16, device=W.device)
+        colsum = torch.empty(N, dtype=torch.float32, device=W.device)
+        cbias = torch.empty(N, dtype=torch.float32, device=W.device)
+        self._check(self.lib.wf_ln_fold(self.handle, W.data_ptr(), ln_g.data_ptr(), ln_b.data_ptr(),
+                                        bias.data_ptr() if bias is not None else None, Wg.data_ptr(), colsum.data_ptr(),
+                                        cbias.data_ptr(), N, K, _stream_ptr(stream)))
+        return Wg, colsum, cbias
+
+    def wf_gemm_ln_bf16(self, x_hi: torch.Tensor, stats: torch.Tensor, Wg: torch.Tensor, colsum: torch.Tensor,
+                        cbias: torch.Tensor, gelu: bool, stream=None):
+        """C bf16 [M, N] = (gelu of) LayerNorm(x) W^T + bias from x_hi, the row statistics of x and folded weights."""
+        M, K = x_hi.shape
+        N = Wg.shape[0]
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=x_hi.device)
+        self._check(self.lib.wf_gemm_ln_bf16(self.handle, x_hi.data_ptr(), stats.data_ptr(), Wg.data_ptr(), colsum.data_ptr(),
+                                             cbias.data_ptr(), out.data_ptr(), M, N, K, 1 if gelu else 0, _stream_ptr(stream)))
+        return out
 
     def wf_cross_kv(self, hidden: torch.Tensor, W_kv: torch.Tensor, b_kv: torch.Tensor, kv_out=None, stream=None):
         """hidden [M, d], W_kv [n_dec * 2 d, d] (path dtype), b_kv float32 [n_dec * 2 d] -> kv [M, n_dec * 2 d]."""

@@ -11,22 +11,20 @@
 
 using namespace wf;
 
-namespace wf {
-static int g_pdl = 1;
-int pdl_enabled() { return g_pdl; }
-void pdl_set(int on) { g_pdl = on; }
-}  // namespace wf
-
 namespace {
 constexpr int kRing = 4;          // per-call metadata slots (pinned host + device)
 constexpr int kMaxTailSamples = 16000;  // longest raw-audio hush word (1 s)
 constexpr int kMinSamples = 401;  // reflect padding of 200 needs more than 200 samples on each side
 }  // namespace
 
+// float32 path: weights as given, LayerNorm parameters applied by the LayerNorm kernel.
+// bf16 path: wqkv and w1 hold W diag(gamma) of the LayerNorm in front of them, bqkv / b1 the
+// bias plus W beta, cs_qkv / cs_1 the row sums of the folded weights (see kEpiLnBias).
 struct LayerW {
   float *ln1_g, *ln1_b, *ln2_g, *ln2_b;
   void *wqkv, *wo, *w1, *w2;
   float *bqkv, *bo, *b1, *b2;
+  float *cs_qkv, *cs_1;
   CUtensorMap tm_wqkv, tm_wo, tm_w1, tm_w2;
 };
 
@@ -52,8 +50,9 @@ struct wf_encoder {
   void *conv1_w, *conv2_w;
   float *conv1_b, *conv2_b, *lnp_g, *lnp_b;
   std::vector<LayerW> layers;
-  CUtensorMap tm_conv1_w, tm_conv2_w, tm_zp, tm_c1p, tm_h, tm_attn, tm_fc1;
-  CUtensorMap tmo_c1p, tmo_qkv, tmo_fc1, tmo_x;  // epilogue outputs
+  CUtensorMap tm_conv1_w, tm_conv2_w, tm_zp, tm_c1p, tm_xh, tm_attn, tm_fc1;
+  CUtensorMap tmo_c1p, tmo_qkv, tmo_fc1;         // epilogue outputs
+  CUtensorMap tmx_hi, tmx_lo;                    // residual stream planes: fetched and stored by the residual epilogue
   CUtensorMap tm_qkv, tm_qkv_kv;                 // attention operand loads (128- and 96-row boxes)
 
   float* logmel;
@@ -61,8 +60,12 @@ struct wf_encoder {
   void *zp_alloc, *c1p;
   int* row_valid;
   int2* row_dst;
-  float* x;
-  void *h, *qkv, *attn, *fc1;
+  float* x;                 // float32 path: residual stream
+  void* h;                  // float32 path: LayerNorm output
+  __nv_bfloat16 *xh, *xl;   // bf16 path: residual stream x = xh + xl
+  float2* stats;            // bf16 path: [d_model / 128][max_tokens] row partial (sum, sum of squares) of x
+  void *qkv, *attn, *fc1;
+  LaunchOpts opt;
   float* audio_stage;
   void* out_stage;
   int* err_flag;
@@ -231,9 +234,14 @@ int build_attn_work(const int* tok, const std::vector<int>& order, bool bf16, in
 
 // Builds prefix sums, the padded-row layout and the work lists for one call into `hm`
 // (host ints), validating every length.  `frames_given`: `len` holds frame counts, not samples.
+// `front_end_only`: the plan of wf_logmel (no hush rows, no token limits, no attention work list).
 wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Plan* p, int* hm,
-                    bool build_work = true, long tail_samples = 0) {
+                    bool front_end_only = false, long tail_samples = 0) {
   const wf_config& c = e->cfg;
+  const bool build_work = !front_end_only;
+  const long hush_rows = front_end_only ? 0 : c.hush_frames;
+  const long n_ctx = front_end_only ? (1L << 28) : c.n_ctx;
+  const long max_tokens = front_end_only ? (1L << 40) : c.max_tokens;
   if (B < 0 || (B > 0 && !len)) return fail(e, WF_ERR_INVALID_ARG, "bad batch size or NULL lengths");
   if (B > c.max_batch) return fail(e, WF_ERR_CAPACITY, "batch %d exceeds max_batch %d", B, c.max_batch);
   MetaLayout& ml = p->ml;
@@ -259,9 +267,9 @@ wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Pl
       if (L < kMinSamples) return fail(e, WF_ERR_TOO_SHORT, "buffer %d has %ld samples (need >= %d)", i, L, kMinSamples);
       T = (L + tail_samples) / kHop;  // a raw-audio hush word lengthens every buffer
     }
-    long rows = T + c.hush_frames;
+    long rows = T + hush_rows;
     long n = (rows + 1) / 2;
-    if (n > c.n_ctx) return fail(e, WF_ERR_TOO_LONG, "sequence %d would have %ld tokens (n_ctx %d)", i, n, c.n_ctx);
+    if (n > n_ctx) return fail(e, WF_ERR_TOO_LONG, "sequence %d would have %ld tokens (n_ctx %d)", i, n, c.n_ctx);
     hm[ml.sample_off + i] = (int)samples;
     hm[ml.frames + i] = (int)T;
     hm[ml.frame_off + i] = (int)frames;
@@ -275,7 +283,7 @@ wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Pl
     tiles += (T + kFeFrames - 1) / kFeFrames;
     max_pr = std::max<int>(max_pr, (int)(2 * (n + 1)));
     if (samples > c.max_samples) return fail(e, WF_ERR_CAPACITY, "more than max_samples=%ld samples", c.max_samples);
-    if (tokens > c.max_tokens) return fail(e, WF_ERR_CAPACITY, "more than max_tokens=%ld tokens", c.max_tokens);
+    if (tokens > max_tokens) return fail(e, WF_ERR_CAPACITY, "more than max_tokens=%ld tokens", c.max_tokens);
   }
   hm[ml.sample_off + B] = (int)samples;
   hm[ml.frames + B] = 0;
@@ -324,19 +332,13 @@ wf_status ring_release(wf_encoder* e, int slot, cudaStream_t s) {
   return WF_OK;
 }
 
-void gemm(wf_encoder* e, const CUtensorMap* ta, const CUtensorMap* tb, const CUtensorMap* tc, const void* A,
-          long lda, const void* W, long ldw, long M, int N, int K, int a_cols, int epi, const EpiParams& ep,
-          cudaStream_t s) {
-  if (e->bf16) launch_gemm_bf16(*ta, *tb, *tc, M, N, K, a_cols, epi, ep, e->err_flag, e->num_sms, s);
-  else launch_gemm_f32((const float*)A, lda, (const float*)W, ldw, M, N, K, epi, ep, s);
-}
-
-// Everything after the log-mel rows sit in the padded-row layout.
-wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidden_out, cudaStream_t s) {
+// Everything after the log-mel rows sit in the padded-row layout, float32 path: SIMT GEMMs, a
+// LayerNorm kernel in front of the QKV and FC1 GEMMs, float32 residual stream.
+wf_status run_encoder_f32(wf_encoder* e, const Plan& p, const int* meta, void* hidden_out, cudaStream_t s) {
   const wf_config& c = e->cfg;
   const int d = c.d_model, F = c.d_mlp;
   const long M = p.total_tokens;
-  const int bf = e->bf16 ? 1 : 0;
+  const float* zp = (const float*)e->zp_alloc;
   {
     Prof pr(e, 1, s);
     launch_build_maps(meta, p.ml, p.B, p.max_prows_seq, c.hush_frames, e->row_valid, e->row_dst, s);
@@ -345,62 +347,134 @@ wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidde
     Prof pr(e, 2, s);
     EpiParams ep{};
     ep.bias = e->conv1_b; ep.out = e->c1p; ep.ldc = d; ep.row_valid = e->row_valid;
-    gemm(e, &e->tm_zp, &e->tm_conv1_w, &e->tmo_c1p, e->zp_alloc, e->mel_ld, e->conv1_w, 3L * e->mel_ld, p.total_prows, d,
-         3 * e->mel_ld, e->mel_ld, kEpiConv1, ep, s);
+    launch_gemm_f32(zp, e->mel_ld, (const float*)e->conv1_w, 3L * e->mel_ld, p.total_prows, d, 3 * e->mel_ld, kEpiConv1, ep, s);
   }
   {
     Prof pr(e, 2, s);
     EpiParams ep{};
     ep.bias = e->conv2_b; ep.resid = e->x; ep.ldc = d; ep.row_dst = e->row_dst; ep.pe = e->pe;
-    gemm(e, &e->tm_c1p, &e->tm_conv2_w, &e->tmo_x, e->c1p, 2L * d, e->conv2_w, 3L * d, p.total_prows / 2, d, 3 * d, 2 * d,
-         kEpiConv2, ep, s);
+    launch_gemm_f32((const float*)e->c1p, 2L * d, (const float*)e->conv2_w, 3L * d, p.total_prows / 2, d, 3 * d, kEpiConv2, ep, s);
   }
   for (int l = 0; l < c.n_layer; ++l) {
     LayerW& w = e->layers[l];
     {
       Prof pr(e, 3, s);
-      launch_layernorm(e->x, w.ln1_g, w.ln1_b, e->h, bf, M, d, s);
+      launch_layernorm(e->x, w.ln1_g, w.ln1_b, (float*)e->h, M, d, s);
     }
     {
       Prof pr(e, 4, s);
       EpiParams ep{};
       ep.bias = w.bqkv; ep.out = e->qkv; ep.ldc = 3L * d;
-      gemm(e, &e->tm_h, &w.tm_wqkv, &e->tmo_qkv, e->h, d, w.wqkv, d, M, 3 * d, d, d, kEpiBias, ep, s);
+      launch_gemm_f32((const float*)e->h, d, (const float*)w.wqkv, d, M, 3 * d, d, kEpiBias, ep, s);
     }
     {
       Prof pr(e, 5, s);
-      if (e->bf16) launch_attention_bf16(e->tm_qkv, e->tm_qkv_kv, (__nv_bfloat16*)e->attn, meta, p.ml, p.n_work, p.n_attn_items, d, e->err_flag, e->num_sms, s);
-      else launch_attention_f32((const float*)e->qkv, (float*)e->attn, meta, p.ml, p.n_work, d, s);
+      launch_attention_f32((const float*)e->qkv, (float*)e->attn, meta, p.ml, p.n_work, d, s);
     }
     {
       Prof pr(e, 4, s);
       EpiParams ep{};
       ep.bias = w.bo; ep.resid = e->x; ep.ldc = d;
-      gemm(e, &e->tm_attn, &w.tm_wo, &e->tmo_x, e->attn, d, w.wo, d, M, d, d, d, kEpiBiasResid, ep, s);
+      launch_gemm_f32((const float*)e->attn, d, (const float*)w.wo, d, M, d, d, kEpiBiasResid, ep, s);
     }
     {
       Prof pr(e, 3, s);
-      launch_layernorm(e->x, w.ln2_g, w.ln2_b, e->h, bf, M, d, s);
+      launch_layernorm(e->x, w.ln2_g, w.ln2_b, (float*)e->h, M, d, s);
     }
     {
       Prof pr(e, 4, s);
       EpiParams ep{};
       ep.bias = w.b1; ep.out = e->fc1; ep.ldc = F;
-      gemm(e, &e->tm_h, &w.tm_w1, &e->tmo_fc1, e->h, d, w.w1, d, M, F, d, d, kEpiBiasGelu, ep, s);
+      launch_gemm_f32((const float*)e->h, d, (const float*)w.w1, d, M, F, d, kEpiBiasGelu, ep, s);
     }
     {
       Prof pr(e, 4, s);
       EpiParams ep{};
       ep.bias = w.b2; ep.resid = e->x; ep.ldc = d;
-      gemm(e, &e->tm_fc1, &w.tm_w2, &e->tmo_x, e->fc1, F, w.w2, F, M, d, F, F, kEpiBiasResid, ep, s);
+      launch_gemm_f32((const float*)e->fc1, F, (const float*)w.w2, F, M, d, F, kEpiBiasResid, ep, s);
     }
   }
   {
     Prof pr(e, 3, s);
-    launch_layernorm(e->x, e->lnp_g, e->lnp_b, hidden_out, bf, M, d, s);
+    launch_layernorm(e->x, e->lnp_g, e->lnp_b, (float*)hidden_out, M, d, s);
   }
   WF_CUDA(e, cudaGetLastError());
   return WF_OK;
+}
+
+// The same on the bf16 path: tcgen05 GEMMs; the residual stream is the pair of bf16 planes
+// (xh, xl); its producers (conv2, out-projection, FC2) leave per-row partial sums in `stats`, from
+// which the QKV and FC1 GEMMs, whose weights carry the LayerNorm's gain, finish the LayerNorm in
+// their epilogues.  Only the final LayerNorm is a kernel of its own.
+wf_status run_encoder_bf16(wf_encoder* e, const Plan& p, const int* meta, void* hidden_out, cudaStream_t s) {
+  const wf_config& c = e->cfg;
+  const int d = c.d_model, F = c.d_mlp;
+  const long M = p.total_tokens;
+  auto gemm = [&](const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2, long m,
+                  int n, int k, int a_cols, int epi, const EpiParams& ep) {
+    launch_gemm_bf16(ta, tb, tc, tc2, m, n, k, a_cols, epi, ep, e->err_flag, e->num_sms, e->opt, s);
+  };
+  {
+    Prof pr(e, 1, s);
+    launch_build_maps(meta, p.ml, p.B, p.max_prows_seq, c.hush_frames, e->row_valid, e->row_dst, s);
+  }
+  {
+    Prof pr(e, 2, s);
+    EpiParams ep{};
+    ep.bias = e->conv1_b; ep.out = e->c1p; ep.ldc = d; ep.row_valid = e->row_valid;
+    gemm(e->tm_zp, e->tm_conv1_w, e->tmo_c1p, e->tmo_c1p, p.total_prows, d, 3 * e->mel_ld, e->mel_ld, kEpiConv1, ep);
+  }
+  {
+    Prof pr(e, 2, s);
+    EpiParams ep{};
+    ep.bias = e->conv2_b; ep.ldc = d; ep.row_dst = e->row_dst; ep.pe = e->pe;
+    ep.x_hi = e->xh; ep.x_lo = e->xl; ep.stats_out = e->stats; ep.stats_pitch = c.max_tokens;
+    gemm(e->tm_c1p, e->tm_conv2_w, e->tmx_hi, e->tmx_lo, p.total_prows / 2, d, 3 * d, 2 * d, kEpiConv2, ep);
+  }
+  for (int l = 0; l < c.n_layer; ++l) {
+    LayerW& w = e->layers[l];
+    {
+      Prof pr(e, 4, s);
+      EpiParams ep{};
+      ep.bias = w.bqkv; ep.colsum = w.cs_qkv; ep.stats_in = e->stats; ep.stats_pitch = c.max_tokens;
+      ep.out = e->qkv; ep.ldc = 3L * d;
+      gemm(e->tm_xh, w.tm_wqkv, e->tmo_qkv, e->tmo_qkv, M, 3 * d, d, d, kEpiLnBias, ep);
+    }
+    {
+      Prof pr(e, 5, s);
+      launch_attention_bf16(e->tm_qkv, e->tm_qkv_kv, (__nv_bfloat16*)e->attn, meta, p.ml, p.n_work, p.n_attn_items, d,
+                            e->err_flag, e->num_sms, e->opt.pdl != 0, s);
+    }
+    {
+      Prof pr(e, 4, s);
+      EpiParams ep{};
+      ep.bias = w.bo; ep.ldc = d; ep.stats_out = e->stats; ep.stats_pitch = c.max_tokens;
+      gemm(e->tm_attn, w.tm_wo, e->tmx_hi, e->tmx_lo, M, d, d, d, kEpiResidSplit, ep);
+    }
+    {
+      Prof pr(e, 4, s);
+      EpiParams ep{};
+      ep.bias = w.b1; ep.colsum = w.cs_1; ep.stats_in = e->stats; ep.stats_pitch = c.max_tokens;
+      ep.out = e->fc1; ep.ldc = F;
+      gemm(e->tm_xh, w.tm_w1, e->tmo_fc1, e->tmo_fc1, M, F, d, d, kEpiLnBiasGelu, ep);
+    }
+    {
+      Prof pr(e, 4, s);
+      EpiParams ep{};
+      ep.bias = w.b2; ep.ldc = d; ep.stats_out = e->stats; ep.stats_pitch = c.max_tokens;
+      gemm(e->tm_fc1, w.tm_w2, e->tmx_hi, e->tmx_lo, M, d, F, F, kEpiResidSplit, ep);
+    }
+  }
+  {
+    Prof pr(e, 3, s);
+    launch_layernorm_split(e->xh, e->xl, e->lnp_g, e->lnp_b, (__nv_bfloat16*)hidden_out, M, d, e->opt.pdl != 0, s);
+  }
+  WF_CUDA(e, cudaGetLastError());
+  return WF_OK;
+}
+
+wf_status run_encoder(wf_encoder* e, const Plan& p, const int* meta, void* hidden_out, cudaStream_t s) {
+  return e->bf16 ? run_encoder_bf16(e, p, meta, hidden_out, s) : run_encoder_f32(e, p, meta, hidden_out, s);
 }
 
 wf_status encode_impl(wf_encoder* e, const float* audio, const float* mel, const long* len, int B,
@@ -416,7 +490,7 @@ wf_status encode_impl(wf_encoder* e, const float* audio, const float* mel, const
   wf_status st = ring_acquire(e, &slot);
   if (st != WF_OK) return st;
   Plan p;
-  st = make_plan(e, len, mel != nullptr, B, &p, e->meta_host[slot], true, tail_len);
+  st = make_plan(e, len, mel != nullptr, B, &p, e->meta_host[slot], false, tail_len);
   if (st == WF_OK && (long)p.total_frames > e->cap_frames)
     st = fail(e, WF_ERR_CAPACITY, "more than %ld frames", e->cap_frames);
   if (st != WF_OK) return st;
@@ -491,15 +565,14 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     if (!tma_api_init(&e->tma)) return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     WF_CUDA(e, gemm_bf16_configure());
     WF_CUDA(e, attention_bf16_configure());
-    // WF_GEMM_TAIL_SPLIT=1 lets residual GEMMs cut the tiles of their last, partial round along K
-    // (faster when M is small; the float32 additions then land in an order that varies from run
-    // to run, so results are no longer bit-reproducible).  Off unless asked for.
+  }
+  WF_CUDA(e, frontend_configure());
+  {
+    // tuning switches, read once per handle
     const char* pdl_env = getenv("WF_PDL");
-    pdl_set(!(pdl_env != nullptr && pdl_env[0] == '0'));
+    e->opt.pdl = !(pdl_env != nullptr && pdl_env[0] == '0');
     const char* small_env = getenv("WF_GEMM_SMALL_TILES");
-    gemm_bf16_set_small_tiles(!(small_env != nullptr && small_env[0] == '0'));
-    const char* split_env = getenv("WF_GEMM_TAIL_SPLIT");
-    gemm_bf16_set_tail_split(split_env != nullptr && split_env[0] == '1');
+    e->opt.small_tiles = !(small_env != nullptr && small_env[0] == '0');
   }
   // tables
   WF_TRY(dev_alloc<float>(e, &e->dft_basis, 2L * kFold * kBasisCols));
@@ -526,24 +599,38 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     return fail(e, WF_ERR_INVALID_ARG, "a per-layer weight array is NULL");
   for (int l = 0; l < c.n_layer; ++l) {
     LayerW& L = e->layers[l];
-    WF_TRY(own_f32(e, &L.ln1_g, w->ln1_g[l], d, s));
-    WF_TRY(own_f32(e, &L.ln1_b, w->ln1_b[l], d, s));
-    WF_TRY(own_f32(e, &L.ln2_g, w->ln2_g[l], d, s));
-    WF_TRY(own_f32(e, &L.ln2_b, w->ln2_b[l], d, s));
+    if (!w->ln1_g[l] || !w->ln1_b[l] || !w->ln2_g[l] || !w->ln2_b[l] || !w->wq[l] || !w->wk[l] || !w->wv[l] ||
+        !w->bq[l] || !w->bv[l] || !w->w1[l] || !w->b1[l])
+      return fail(e, WF_ERR_INVALID_ARG, "a weight pointer of layer %d is NULL", l);
     WF_TRY(dev_alloc_bytes(e, &L.wqkv, (size_t)3 * d * d * e->esz));
-    WF_TRY(own_mat(e, L.wqkv, 0, w->wq[l], (size_t)d * d, s));
-    WF_TRY(own_mat(e, L.wqkv, (size_t)d * d, w->wk[l], (size_t)d * d, s));
-    WF_TRY(own_mat(e, L.wqkv, (size_t)2 * d * d, w->wv[l], (size_t)d * d, s));
-    WF_TRY(dev_alloc<float>(e, &L.bqkv, 3 * d, true));  // the key part stays zero
-    if (!w->bq[l] || !w->bv[l]) return fail(e, WF_ERR_INVALID_ARG, "a bias pointer is NULL");
-    WF_CUDA(e, cudaMemcpyAsync(L.bqkv, w->bq[l], d * sizeof(float), cudaMemcpyDeviceToDevice, s));
-    WF_CUDA(e, cudaMemcpyAsync(L.bqkv + 2 * d, w->bv[l], d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    WF_TRY(dev_alloc<float>(e, &L.bqkv, 3 * d, true));  // float32 path: the key part stays zero
+    WF_TRY(dev_alloc_bytes(e, &L.w1, (size_t)F * d * e->esz));
+    if (e->bf16) {
+      // LayerNorm 1 folded into the QKV weight, LayerNorm 2 into FC1's
+      WF_TRY(dev_alloc<float>(e, &L.cs_qkv, 3 * d));
+      WF_TRY(dev_alloc<float>(e, &L.cs_1, F));
+      WF_TRY(dev_alloc<float>(e, &L.b1, F));
+      __nv_bfloat16* wqkv = (__nv_bfloat16*)L.wqkv;
+      launch_ln_fold(w->wq[l], w->ln1_g[l], w->ln1_b[l], w->bq[l], wqkv, L.cs_qkv, L.bqkv, d, d, s);
+      launch_ln_fold(w->wk[l], w->ln1_g[l], w->ln1_b[l], nullptr, wqkv + (size_t)d * d, L.cs_qkv + d, L.bqkv + d, d, d, s);
+      launch_ln_fold(w->wv[l], w->ln1_g[l], w->ln1_b[l], w->bv[l], wqkv + (size_t)2 * d * d, L.cs_qkv + 2 * d, L.bqkv + 2 * d, d, d, s);
+      launch_ln_fold(w->w1[l], w->ln2_g[l], w->ln2_b[l], w->b1[l], (__nv_bfloat16*)L.w1, L.cs_1, L.b1, F, d, s);
+    } else {
+      WF_TRY(own_f32(e, &L.ln1_g, w->ln1_g[l], d, s));
+      WF_TRY(own_f32(e, &L.ln1_b, w->ln1_b[l], d, s));
+      WF_TRY(own_f32(e, &L.ln2_g, w->ln2_g[l], d, s));
+      WF_TRY(own_f32(e, &L.ln2_b, w->ln2_b[l], d, s));
+      WF_TRY(own_mat(e, L.wqkv, 0, w->wq[l], (size_t)d * d, s));
+      WF_TRY(own_mat(e, L.wqkv, (size_t)d * d, w->wk[l], (size_t)d * d, s));
+      WF_TRY(own_mat(e, L.wqkv, (size_t)2 * d * d, w->wv[l], (size_t)d * d, s));
+      WF_CUDA(e, cudaMemcpyAsync(L.bqkv, w->bq[l], d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+      WF_CUDA(e, cudaMemcpyAsync(L.bqkv + 2 * d, w->bv[l], d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+      WF_TRY(own_mat(e, L.w1, 0, w->w1[l], (size_t)F * d, s));
+      WF_TRY(own_f32(e, &L.b1, w->b1[l], F, s));
+    }
     WF_TRY(dev_alloc_bytes(e, &L.wo, (size_t)d * d * e->esz));
     WF_TRY(own_mat(e, L.wo, 0, w->wo[l], (size_t)d * d, s));
     WF_TRY(own_f32(e, &L.bo, w->bo[l], d, s));
-    WF_TRY(dev_alloc_bytes(e, &L.w1, (size_t)F * d * e->esz));
-    WF_TRY(own_mat(e, L.w1, 0, w->w1[l], (size_t)F * d, s));
-    WF_TRY(own_f32(e, &L.b1, w->b1[l], F, s));
     WF_TRY(dev_alloc_bytes(e, &L.w2, (size_t)d * F * e->esz));
     WF_TRY(own_mat(e, L.w2, 0, w->w2[l], (size_t)d * F, s));
     WF_TRY(own_f32(e, &L.b2, w->b2[l], d, s));
@@ -557,8 +644,14 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
   WF_TRY(dev_alloc_bytes(e, &e->c1p, (size_t)(e->cap_prows + 4) * d * e->esz, true));
   WF_TRY(dev_alloc<int>(e, &e->row_valid, (size_t)e->cap_prows + 4, true));
   WF_TRY(dev_alloc<int2>(e, &e->row_dst, (size_t)e->cap_prows / 2 + 4, true));
-  WF_TRY(dev_alloc<float>(e, &e->x, mt * d));
-  WF_TRY(dev_alloc_bytes(e, &e->h, mt * d * e->esz, true));
+  if (e->bf16) {
+    WF_TRY(dev_alloc<__nv_bfloat16>(e, &e->xh, mt * d, true));
+    WF_TRY(dev_alloc<__nv_bfloat16>(e, &e->xl, mt * d, true));
+    WF_TRY(dev_alloc<float2>(e, &e->stats, (size_t)(d / 128) * mt, true));
+  } else {
+    WF_TRY(dev_alloc<float>(e, &e->x, mt * d));
+    WF_TRY(dev_alloc_bytes(e, &e->h, mt * d * e->esz, true));
+  }
   WF_TRY(dev_alloc_bytes(e, &e->qkv, mt * 3 * d * e->esz, true));
   WF_TRY(dev_alloc_bytes(e, &e->attn, mt * d * e->esz, true));
   WF_TRY(dev_alloc_bytes(e, &e->fc1, mt * F * e->esz, true));
@@ -579,7 +672,7 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     bool ok = true;
     ok &= make_tmap_bf16(e->tma, &e->tm_zp, e->zp_alloc, e->mel_ld, e->cap_prows + 4, e->mel_ld, 128);
     ok &= make_tmap_bf16(e->tma, &e->tm_c1p, e->c1p, 2 * d, (e->cap_prows + 4) / 2, 2 * d, 128);
-    ok &= make_tmap_bf16(e->tma, &e->tm_h, e->h, d, mt, d, 128);
+    ok &= make_tmap_bf16(e->tma, &e->tm_xh, e->xh, d, mt, d, 128);
     ok &= make_tmap_bf16(e->tma, &e->tm_attn, e->attn, d, mt, d, 128);
     ok &= make_tmap_bf16(e->tma, &e->tm_fc1, e->fc1, F, mt, F, 128);
     ok &= make_tmap_bf16(e->tma, &e->tm_qkv, e->qkv, 3 * d, mt, 3 * d, 128);
@@ -587,8 +680,9 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     ok &= make_tmap_out(e->tma, &e->tmo_c1p, e->c1p, 2, d, e->cap_prows + 4);
     ok &= make_tmap_out(e->tma, &e->tmo_qkv, e->qkv, 2, 3 * d, mt);
     ok &= make_tmap_out(e->tma, &e->tmo_fc1, e->fc1, 2, F, mt);
-    ok &= make_tmap_out(e->tma, &e->tmo_x, e->x, 4, d, mt);
-    const uint32_t wbox = gemm_bf16_uses_pair() ? 128 : 256;
+    ok &= make_tmap_out(e->tma, &e->tmx_hi, e->xh, 2, d, mt);
+    ok &= make_tmap_out(e->tma, &e->tmx_lo, e->xl, 2, d, mt);
+    const uint32_t wbox = 128;
     ok &= make_tmap_bf16(e->tma, &e->tm_conv1_w, e->conv1_w, 3 * e->mel_ld, d, 3 * e->mel_ld, wbox);
     ok &= make_tmap_bf16(e->tma, &e->tm_conv2_w, e->conv2_w, 3 * d, d, 3 * d, wbox);
     for (int l = 0; l < c.n_layer; ++l) {
@@ -632,12 +726,7 @@ wf_status wf_logmel(wf_encoder* e, const float* audio, const long* lengths, int 
   if (st != WF_OK) return st;
   Plan p;
   // frame counts do not depend on the hush length; token limits do not apply to the front end
-  wf_config saved = e->cfg;
-  e->cfg.hush_frames = 0;
-  e->cfg.n_ctx = 1 << 28;
-  e->cfg.max_tokens = 1L << 40;
-  st = make_plan(e, lengths, false, B, &p, e->meta_host[slot], false);
-  e->cfg = saved;
+  st = make_plan(e, lengths, false, B, &p, e->meta_host[slot], true);
   if (st != WF_OK) return st;
   if (frames_out)
     for (int i = 0; i < B; ++i) frames_out[i] = e->meta_host[slot][p.ml.frames + i];
@@ -745,19 +834,79 @@ wf_status wf_gemm_bf16(wf_encoder* e, const void* A, const void* W, const float*
                        int K, int mode, void* stream) {
   if (!e) return WF_ERR_INVALID_ARG;
   if (!e->bf16) return fail(e, WF_ERR_INVALID_ARG, "wf_gemm_bf16 needs an encoder created with WF_BF16");
-  if (!A || !W || !bias || !C || M < 0 || N <= 0 || K <= 0 || N % 8 || K % 8 || mode < 0 || mode > 2 ||
+  if (!A || !W || !bias || !C || M < 0 || N <= 0 || K <= 0 || N % 8 || K % 8 || mode < 0 || mode > 1 ||
       ((uintptr_t)A & 15) || ((uintptr_t)W & 15) || ((uintptr_t)C & 15) || ((uintptr_t)bias & 15))
     return fail(e, WF_ERR_INVALID_ARG, "wf_gemm_bf16: bad pointer, size or mode");
   if (M == 0) return WF_OK;
   CUtensorMap ta, tb, tc;
-  if (!make_tmap_bf16(e->tma, &ta, A, K, M, K, 128) || !make_tmap_bf16(e->tma, &tb, W, K, N, K, gemm_bf16_uses_pair() ? 128 : 256) ||
-      !make_tmap_out(e->tma, &tc, C, mode == 2 ? 4 : 2, N, M))
+  if (!make_tmap_bf16(e->tma, &ta, A, K, M, K, 128) || !make_tmap_bf16(e->tma, &tb, W, K, N, K, 128) ||
+      !make_tmap_out(e->tma, &tc, C, 2, N, M))
     return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
   EpiParams ep{};
   ep.bias = bias;
   ep.ldc = N;
-  if (mode == 2) ep.resid = (float*)C; else ep.out = C;
-  launch_gemm_bf16(ta, tb, tc, M, N, K, K, mode, ep, e->err_flag, e->num_sms, (cudaStream_t)stream);
+  ep.out = C;
+  launch_gemm_bf16(ta, tb, tc, tc, M, N, K, K, mode == 0 ? kEpiBias : kEpiBiasGelu, ep, e->err_flag, e->num_sms, e->opt,
+                   (cudaStream_t)stream);
+  WF_CUDA(e, cudaGetLastError());
+  return WF_OK;
+}
+
+wf_status wf_gemm_resid_bf16(wf_encoder* e, const void* A, const void* W, const float* bias, void* x_hi, void* x_lo,
+                             float* stats, long M, int N, int K, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  if (!e->bf16) return fail(e, WF_ERR_INVALID_ARG, "wf_gemm_resid_bf16 needs an encoder created with WF_BF16");
+  if (!A || !W || !bias || !x_hi || !x_lo || !stats || M < 0 || N <= 0 || K <= 0 || N % 128 || K % 8 ||
+      ((uintptr_t)A & 15) || ((uintptr_t)W & 15) || ((uintptr_t)x_hi & 15) || ((uintptr_t)x_lo & 15) ||
+      ((uintptr_t)bias & 15) || ((uintptr_t)stats & 7))
+    return fail(e, WF_ERR_INVALID_ARG, "wf_gemm_resid_bf16: bad pointer or size (N must be a multiple of 128)");
+  if (M == 0) return WF_OK;
+  CUtensorMap ta, tb, th, tl;
+  if (!make_tmap_bf16(e->tma, &ta, A, K, M, K, 128) || !make_tmap_bf16(e->tma, &tb, W, K, N, K, 128) ||
+      !make_tmap_out(e->tma, &th, x_hi, 2, N, M) || !make_tmap_out(e->tma, &tl, x_lo, 2, N, M))
+    return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
+  EpiParams ep{};
+  ep.bias = bias;
+  ep.ldc = N;
+  ep.stats_out = (float2*)stats;
+  ep.stats_pitch = M;
+  launch_gemm_bf16(ta, tb, th, tl, M, N, K, K, kEpiResidSplit, ep, e->err_flag, e->num_sms, e->opt, (cudaStream_t)stream);
+  WF_CUDA(e, cudaGetLastError());
+  return WF_OK;
+}
+
+wf_status wf_ln_fold(wf_encoder* e, const float* W, const float* ln_g, const float* ln_b, const float* bias, void* Wg,
+                     float* colsum, float* cbias, int N, int K, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  if (!W || !ln_g || !ln_b || !Wg || !colsum || !cbias || N <= 0 || K <= 0)
+    return fail(e, WF_ERR_INVALID_ARG, "wf_ln_fold: bad pointer or size");
+  launch_ln_fold(W, ln_g, ln_b, bias, (__nv_bfloat16*)Wg, colsum, cbias, N, K, (cudaStream_t)stream);
+  WF_CUDA(e, cudaGetLastError());
+  return WF_OK;
+}
+
+wf_status wf_gemm_ln_bf16(wf_encoder* e, const void* x_hi, const float* stats, const void* Wg, const float* colsum,
+                          const float* cbias, void* C, long M, int N, int K, int gelu, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  if (!e->bf16) return fail(e, WF_ERR_INVALID_ARG, "wf_gemm_ln_bf16 needs an encoder created with WF_BF16");
+  if (!x_hi || !stats || !Wg || !colsum || !cbias || !C || M < 0 || N <= 0 || K <= 0 || N % 8 || K % 128 ||
+      ((uintptr_t)x_hi & 15) || ((uintptr_t)Wg & 15) || ((uintptr_t)C & 15) || ((uintptr_t)colsum & 15) ||
+      ((uintptr_t)cbias & 15) || ((uintptr_t)stats & 7))
+    return fail(e, WF_ERR_INVALID_ARG, "wf_gemm_ln_bf16: bad pointer or size (K must be a multiple of 128)");
+  if (M == 0) return WF_OK;
+  CUtensorMap ta, tb, tc;
+  if (!make_tmap_bf16(e->tma, &ta, x_hi, K, M, K, 128) || !make_tmap_bf16(e->tma, &tb, Wg, K, N, K, 128) ||
+      !make_tmap_out(e->tma, &tc, C, 2, N, M))
+    return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
+  EpiParams ep{};
+  ep.bias = cbias;
+  ep.colsum = colsum;
+  ep.stats_in = (const float2*)stats;
+  ep.stats_pitch = M;
+  ep.ldc = N;
+  ep.out = C;
+  launch_gemm_bf16(ta, tb, tc, tc, M, N, K, K, gelu ? kEpiLnBiasGelu : kEpiLnBias, ep, e->err_flag, e->num_sms, e->opt,
+                   (cudaStream_t)stream);
   WF_CUDA(e, cudaGetLastError());
   return WF_OK;
 }
@@ -974,10 +1123,10 @@ wf_status wf_cross_kv(wf_encoder* e, const void* hidden, const void* W_kv, const
       return fail(e, WF_ERR_INVALID_ARG, "wf_cross_kv: pointers must be 16-byte aligned");
     CUtensorMap ta, tb, tc;
     if (!make_tmap_bf16(e->tma, &ta, hidden, d, M, d, 128) ||
-        !make_tmap_bf16(e->tma, &tb, W_kv, d, N, d, gemm_bf16_uses_pair() ? 128 : 256) ||
+        !make_tmap_bf16(e->tma, &tb, W_kv, d, N, d, 128) ||
         !make_tmap_out(e->tma, &tc, kv, 2, N, M))
       return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected a tensor map");
-    launch_gemm_bf16(ta, tb, tc, M, N, d, d, kEpiBias, ep, e->err_flag, e->num_sms, (cudaStream_t)stream);
+    launch_gemm_bf16(ta, tb, tc, tc, M, N, d, d, kEpiBias, ep, e->err_flag, e->num_sms, e->opt, (cudaStream_t)stream);
   } else {
     launch_gemm_f32((const float*)hidden, d, (const float*)W_kv, d, M, N, d, kEpiBias, ep, (cudaStream_t)stream);
   }
@@ -1055,7 +1204,8 @@ wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, in
       if (!make_tmap_bf16(e->tma, &tq, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 128) ||
           !make_tmap_bf16(e->tma, &tkv, qkv, 3 * e->cfg.d_model, cu_seqlens[B], 3 * e->cfg.d_model, 96))
         return fail(e, WF_ERR_CUDA, "cuTensorMapEncodeTiled rejected the qkv tensor map");
-      launch_attention_bf16(tq, tkv, (__nv_bfloat16*)out, e->meta_dev[slot], ml, nw, n_items, e->cfg.d_model, e->err_flag, e->num_sms, s);
+      launch_attention_bf16(tq, tkv, (__nv_bfloat16*)out, e->meta_dev[slot], ml, nw, n_items, e->cfg.d_model, e->err_flag, e->num_sms,
+                            e->opt.pdl != 0, s);
     }
     else launch_attention_f32((const float*)qkv, (float*)out, e->meta_dev[slot], ml, nw, e->cfg.d_model, s);
   }

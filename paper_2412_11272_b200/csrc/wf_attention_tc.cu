@@ -537,11 +537,11 @@ cudaError_t attention_bf16_configure() {
 
 void launch_attention_bf16(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, __nv_bfloat16* out,
                            const int* meta, MetaLayout ml, int n_entries, int n_items, int d_model, int* err_flag,
-                           int num_sms, cudaStream_t s) {
+                           int num_sms, bool pdl, cudaStream_t s) {
   if (n_items <= 0) return;
   const int n_head = d_model / kHeadDim;
   const int grid = n_items < num_sms ? n_items : num_sms;
-  launch_dependent(attention_tc_kernel, dim3(grid), dim3(kAttnThreads), kAttnSmem, s, 1, tmap_q, tmap_kv, out, meta, ml,
+  launch_dependent(attention_tc_kernel, dim3(grid), dim3(kAttnThreads), kAttnSmem, s, 1, pdl, tmap_q, tmap_kv, out, meta, ml,
                    n_items, n_entries, n_head, d_model, err_flag);
 }
 

@@ -260,17 +260,18 @@ __global__ void __launch_bounds__(256) frontend_kernel(
   if (lane == 0 && mx > -INFINITY) atomicMax(seq_max + seq, float_to_ordered(mx));
 }
 
+constexpr int kFeSmemBytes = (kFeSmemFloats + 2 * 2 * kBasisChunk * kBasisCols + kFeSpan + 1) * (int)sizeof(float);  // 172,992 B
+
+// Function attributes are per device: called by every create, on the device that is current then.
+cudaError_t frontend_configure() {
+  return cudaFuncSetAttribute(frontend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFeSmemBytes);
+}
+
 void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, int n_tiles,
                      const float* dft_basis, const float* mel_fb_t, int n_mel, float* logmel,
                      int* seq_max, const float* tail, int tail_len, cudaStream_t s) {
-  const int smem = (kFeSmemFloats + 2 * 2 * kBasisChunk * kBasisCols + kFeSpan + 1) * (int)sizeof(float);  // 172,992 B
-  static bool configured = false;
-  if (!configured) {
-    cudaFuncSetAttribute(frontend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    configured = true;
-  }
   if (n_tiles > 0)
-    frontend_kernel<<<n_tiles, 256, smem, s>>>(audio, meta, ml, B, dft_basis, mel_fb_t, n_mel, logmel,
+    frontend_kernel<<<n_tiles, 256, kFeSmemBytes, s>>>(audio, meta, ml, B, dft_basis, mel_fb_t, n_mel, logmel,
                                                 seq_max, tail, tail_len);
 }
 

@@ -7,9 +7,11 @@
 //               accumulation in TMEM) and commits stage releases / accumulator readiness;
 //   warps 2..5  read the accumulator with tcgen05.ld (one row per thread), apply the fused
 //               epilogue, stage 32-row x 128-byte pieces in swizzled shared memory and hand them
-//               to TMA: a tile store for bf16 outputs, a float32 add-reduction (performed at the
-//               L2) for the residual update, so the residual is never read by the SM.  This runs
-//               while the MMA warp already fills the other accumulator buffer.
+//               to TMA for the store.  The residual update fetches the old values of the residual
+//               stream by TMA one piece ahead, adds in place in shared memory and stores from
+//               there, leaving per-row partial sums for the LayerNorm that the next GEMM folds
+//               into its own epilogue.  All this runs while the MMA warp already fills the other
+//               accumulator buffer.
 // Every mbarrier wait is bounded; on a timeout the CTA sets an error word, drains its own
 // TMA copies, frees its tensor memory and returns.
 #include <algorithm>
@@ -25,108 +27,151 @@ using namespace ptx;
 constexpr int kBM = 128;
 constexpr int kBK = 64;
 constexpr int kGemmThreads = 192;
+// Residual epilogue (kEpiResidSplit): every epilogue warp owns kXSets staging sets of 8 KB (a
+// 32-row x 64-column piece of x_hi and of x_lo); the old values of piece p + kXLook are fetched
+// by TMA while piece p is processed, and a set is stored from in place.
+constexpr int kXSets = 2;
+constexpr int kXLook = 1;
+constexpr int kSmemBudget = 224 * 1024;  // operand stages + epilogue staging
 
-template <int BN>
-struct GemmCfg {
-  static constexpr int kStages = BN == 256 ? 4 : 6;
+// Shared-memory plan of a CTA that stages 128 x 64 of A and BROWS x 64 of W per stage.
+template <int BROWS, int EPI>
+struct SmemPlan {
   static constexpr int kABytes = kBM * kBK * 2;
-  static constexpr int kBBytes = BN * kBK * 2;
+  static constexpr int kBBytes = BROWS * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStagingOffset = kStages * kStageBytes;       // 4 warps x 2 buffers x 4 KB
-  static constexpr int kStagingBytes = 4 * 2 * 4096;
-  static constexpr int kBarOffset = kStagingOffset + kStagingBytes;
-  static constexpr int kSmemBytes = kBarOffset + 256 + 1024;  // barriers + alignment slack
-  static constexpr int kTmemCols = 2 * BN;
+  static constexpr int kStagingPerWarp = EPI == kEpiResidSplit ? kXSets * 8192 : 2 * 4096;
+  static constexpr int kStages = (kSmemBudget - 4 * kStagingPerWarp) / kStageBytes;
+  static constexpr int kStagingOffset = kStages * kStageBytes;
+  static constexpr int kBarOffset = kStagingOffset + 4 * kStagingPerWarp;
+  // barriers: full[kStages], empty[kStages], tfull[2], tempty[2], xld[4][kXSets]; then the tensor
+  // memory slot and the abort flag
+  static constexpr int kNumBars = 2 * kStages + 4 + 4 * kXSets;
+  static constexpr int kSmemBytes = kBarOffset + 8 * kNumBars + 16 + 1024;  // + alignment slack
+  static_assert(kStages >= 3 && 8 * kNumBars + 16 <= 256, "shared-memory plan");
 };
+constexpr int kMaxGemmSmem = kSmemBudget + 256 + 1024;
 
-// bias add (+ GELU) of 32 accumulator columns starting at col0 (col0 + 32 <= padded N is not
-// required: columns at or beyond N are computed from a clamped bias index and never stored).
+__host__ __device__ constexpr bool epi_is_ln(int epi) { return epi == kEpiLnBias || epi == kEpiLnBiasGelu; }
+
+// Mean and reciprocal standard deviation of one row of x (K columns) from the partial sums its
+// producer left: returns (rstd, -rstd * mean).
+__device__ __forceinline__ float2 row_norm(const EpiParams& ep, long row, long M, int K) {
+  float s1 = 0.f, s2 = 0.f;
+  if (row < M) {
+    for (int p = 0; p < K / 128; ++p) {
+      const float2 t = __ldg(ep.stats_in + (long)p * ep.stats_pitch + row);
+      s1 += t.x;
+      s2 += t.y;
+    }
+  }
+  const float inv = 1.0f / (float)K;
+  const float mean = s1 * inv;
+  const float var = fmaxf(fmaf(s2, inv, -mean * mean), 0.f);
+  const float rstd = rsqrtf(var + 1e-5f);
+  return make_float2(rstd, -rstd * mean);
+}
+
+// Epilogue arithmetic of 32 accumulator columns starting at col0 (col0 + 32 <= padded N is not
+// required: columns at or beyond N are computed from zeros and never stored).  nrm = row_norm()
+// for the LayerNorm-folded epilogues.
 template <int EPI>
 __device__ __forceinline__ void bias_act32(const EpiParams& ep, int col0, int N, const uint32_t (&acc)[32],
-                                           float (&v)[32], bool with_bias = true) {
+                                           float (&v)[32], float2 nrm) {
+  const uint64_t rs = pack_f32x2(nrm.x, nrm.x), nm = pack_f32x2(nrm.y, nrm.y);
 #pragma unroll
   for (int g = 0; g < 8; ++g) {
-    int col = col0 + 4 * g;
-    float4 b = (col < N && with_bias) ? __ldg(reinterpret_cast<const float4*>(ep.bias + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    unpack_f32x2(add_f32x2(pack_f32x2(__uint_as_float(acc[4 * g + 0]), __uint_as_float(acc[4 * g + 1])),
-                           pack_f32x2(b.x, b.y)), v[4 * g + 0], v[4 * g + 1]);
-    unpack_f32x2(add_f32x2(pack_f32x2(__uint_as_float(acc[4 * g + 2]), __uint_as_float(acc[4 * g + 3])),
-                           pack_f32x2(b.z, b.w)), v[4 * g + 2], v[4 * g + 3]);
+    const int col = col0 + 4 * g;
+    const float4 b = col < N ? __ldg(reinterpret_cast<const float4*>(ep.bias + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    const uint64_t a01 = pack_f32x2(__uint_as_float(acc[4 * g + 0]), __uint_as_float(acc[4 * g + 1]));
+    const uint64_t a23 = pack_f32x2(__uint_as_float(acc[4 * g + 2]), __uint_as_float(acc[4 * g + 3]));
+    if (epi_is_ln(EPI)) {
+      const float4 cs = col < N ? __ldg(reinterpret_cast<const float4*>(ep.colsum + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      unpack_f32x2(fma_f32x2(rs, a01, fma_f32x2(nm, pack_f32x2(cs.x, cs.y), pack_f32x2(b.x, b.y))), v[4 * g + 0], v[4 * g + 1]);
+      unpack_f32x2(fma_f32x2(rs, a23, fma_f32x2(nm, pack_f32x2(cs.z, cs.w), pack_f32x2(b.z, b.w))), v[4 * g + 2], v[4 * g + 3]);
+    } else {
+      unpack_f32x2(add_f32x2(a01, pack_f32x2(b.x, b.y)), v[4 * g + 0], v[4 * g + 1]);
+      unpack_f32x2(add_f32x2(a23, pack_f32x2(b.z, b.w)), v[4 * g + 2], v[4 * g + 3]);
+    }
   }
-  if (EPI == kEpiBiasGelu || EPI == kEpiConv1 || EPI == kEpiConv2) {
+  if (EPI == kEpiBiasGelu || EPI == kEpiLnBiasGelu || EPI == kEpiConv1 || EPI == kEpiConv2) {
 #pragma unroll
     for (int i = 0; i < 32; i += 2) gelu_sigmoid_poly2(v[i], v[i + 1]);
   }
 }
 
-// Direct (non-TMA) store of one row segment for the stride-2 conv epilogue, whose output rows
-// are remapped per sequence: resid[dst] = gelu(acc + bias) + pe[pos].
-__device__ __forceinline__ void conv2_store32(const EpiParams& ep, long row, long M, int col0, int N,
-                                              const float (&v)[32]) {
-  if (row >= M || col0 >= N) return;
-  int2 d = ep.row_dst[row];
-  if (d.x < 0) return;
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi): two values per call, packed as bf16 pairs
+// (first value in the low half).
+__device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  hi = *reinterpret_cast<uint32_t*>(&h);
+  __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __uint_as_float(hi << 16), x1 - __uint_as_float(hi & 0xffff0000u));
+  lo = *reinterpret_cast<uint32_t*>(&l);
+}
+
+// Stride-2 conv epilogue, whose output rows are remapped per sequence (plain stores, no TMA):
+// x[dst] = gelu(acc + bias) + pe[pos], written as the two planes of the residual stream; s1 / s2
+// gather the row's sum and sum of squares.
+__device__ __forceinline__ void conv2_store32(const EpiParams& ep, int2 d, int col0, int N, const float (&v)[32],
+                                              float& s1, float& s2) {
+  if (d.x < 0 || col0 >= N) return;
 #pragma unroll
-  for (int g = 0; g < 8; ++g) {
-    int col = col0 + 4 * g;
+  for (int g = 0; g < 4; ++g) {
+    const int col = col0 + 8 * g;
     if (col >= N) break;
-    float4 e = __ldg(reinterpret_cast<const float4*>(ep.pe + (long)d.y * ep.ldc + col));
-    *reinterpret_cast<float4*>(ep.resid + (long)d.x * ep.ldc + col) =
-        make_float4(v[4 * g] + e.x, v[4 * g + 1] + e.y, v[4 * g + 2] + e.z, v[4 * g + 3] + e.w);
+    const float4 e0 = __ldg(reinterpret_cast<const float4*>(ep.pe + (long)d.y * ep.ldc + col));
+    const float4 e1 = __ldg(reinterpret_cast<const float4*>(ep.pe + (long)d.y * ep.ldc + col + 4));
+    const float x[8] = {v[8 * g] + e0.x,     v[8 * g + 1] + e0.y, v[8 * g + 2] + e0.z, v[8 * g + 3] + e0.w,
+                        v[8 * g + 4] + e1.x, v[8 * g + 5] + e1.y, v[8 * g + 6] + e1.z, v[8 * g + 7] + e1.w};
+    uint4 h, l;
+    split_bf16x2(x[0], x[1], h.x, l.x);
+    split_bf16x2(x[2], x[3], h.y, l.y);
+    split_bf16x2(x[4], x[5], h.z, l.z);
+    split_bf16x2(x[6], x[7], h.w, l.w);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      s1 += x[i];
+      s2 = fmaf(x[i], x[i], s2);
+    }
+    *reinterpret_cast<uint4*>(ep.x_hi + (long)d.x * ep.ldc + col) = h;
+    *reinterpret_cast<uint4*>(ep.x_lo + (long)d.x * ep.ldc + col) = l;
   }
 }
 
 // Epilogue of one 128 x BN accumulator tile for the warp that owns TMEM lanes 32 * quarter ..:
 // t_row is the tensor-memory address of that lane group's first column of the tile, m0 / n0 the
-// tile origin in the output, stage_base this warp's two 4 KB staging buffers.
-template <int BN, int EPI, int NBUF = 2>
+// tile origin in the output, stage_base this warp's staging buffers (bf16 outputs: two of 4 KB).
+template <int BN, int EPI>
 __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtensorMap* tmap_c, uint32_t t_row, int m0,
-                                              int n0, long M, int N, int quarter, int lane, uint32_t stage_base,
-                                              uint32_t& piece, bool with_bias = true) {
+                                              int n0, long M, int N, int K, int quarter, int lane, uint32_t stage_base,
+                                              uint32_t& piece) {
   const long row = (long)m0 + quarter * 32 + lane;
   if (EPI == kEpiConv2) {
+    const int2 d = row < M ? ep.row_dst[row] : make_int2(-1, 0);
+    float s1 = 0.f, s2 = 0.f;
 #pragma unroll 1
     for (int c = 0; c < BN / 32; ++c) {
       uint32_t a32[32];
       float v[32];
       tmem_ld_32x32(t_row + c * 32, a32);
       tmem_ld_wait();
-      bias_act32<EPI>(ep, n0 + c * 32, N, a32, v);
-      conv2_store32(ep, row, M, n0 + c * 32, N, v);
-    }
-  } else if (EPI == kEpiBiasResid) {
-    // float32: 32 columns = 128 bytes per row and piece
-#pragma unroll 1
-    for (int c = 0; c < BN / 32; ++c) {
-      const uint32_t buf = stage_base + (uint32_t)((piece % NBUF) * 4096);
-      if (lane == 0) bulk_wait_read<NBUF - 1>();   // the copy that last read this buffer is done with it
-      __syncwarp();
-      uint32_t a32[32];
-      float v[32];
-      tmem_ld_32x32(t_row + c * 32, a32);
-      tmem_ld_wait();
-      bias_act32<EPI>(ep, n0 + c * 32, N, a32, v, with_bias);
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        st_shared_v4(buf + lane * 128 + ((j ^ (lane & 7)) << 4), __float_as_uint(v[4 * j]),
-                     __float_as_uint(v[4 * j + 1]), __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) {
-        if (n0 + c * 32 < N && (long)m0 + quarter * 32 < M) tma_reduce_add_2d(tmap_c, buf, n0 + c * 32, m0 + quarter * 32);
-        bulk_commit();  // one group per piece, empty when the piece lies outside the matrix: wait_read<1>
-                        // above counts groups to know that the copy two pieces back has let go of its buffer
+      bias_act32<EPI>(ep, n0 + c * 32, N, a32, v, make_float2(0.f, 0.f));
+      conv2_store32(ep, d, n0 + c * 32, N, v, s1, s2);
+      if ((c & 3) == 3) {  // 128 columns done: one partial of the row statistics
+        if (d.x >= 0 && n0 + c * 32 < N) ep.stats_out[(long)((n0 + c * 32) >> 7) * ep.stats_pitch + d.x] = make_float2(s1, s2);
+        s1 = s2 = 0.f;
       }
-      ++piece;
     }
   } else {
     // bf16: 64 columns = 128 bytes per row and piece
     bool valid = true;
     if (EPI == kEpiConv1) valid = row < M && ep.row_valid[row] != 0;
+    float2 nrm = make_float2(0.f, 0.f);
+    if (epi_is_ln(EPI)) nrm = row_norm(ep, row, M, K);
 #pragma unroll 1
     for (int c = 0; c < BN / 64; ++c) {
-      const uint32_t buf = stage_base + (uint32_t)((piece % NBUF) * 4096);
-      if (lane == 0) bulk_wait_read<NBUF - 1>();
+      const uint32_t buf = stage_base + (uint32_t)((piece & 1u) * 4096);
+      if (lane == 0) bulk_wait_read<1>();   // the copy that last read this buffer is done with it
       __syncwarp();
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
@@ -134,7 +179,7 @@ __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtenso
         float v[32];
         tmem_ld_32x32(t_row + c * 64 + hf * 32, a32);
         tmem_ld_wait();
-        bias_act32<EPI>(ep, n0 + c * 64 + hf * 32, N, a32, v);
+        bias_act32<EPI>(ep, n0 + c * 64 + hf * 32, N, a32, v, nrm);
         if (EPI == kEpiConv1 && !valid) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = 0.f;
@@ -154,18 +199,143 @@ __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtenso
       __syncwarp();
       if (lane == 0) {
         if (n0 + c * 64 < N && (long)m0 + quarter * 32 < M) tma_store_2d(tmap_c, buf, n0 + c * 64, m0 + quarter * 32);
-        bulk_commit();  // one group per piece, also when nothing was stored (see above)
+        // One bulk group per piece, empty when the piece lies outside the matrix: wait_read<1> above
+        // counts groups to know that the copy two pieces back has let go of its buffer.
+        bulk_commit();
       }
       ++piece;
     }
   }
 }
 
+// ---- residual epilogue on the split residual stream --------------------------------------------
+// The pieces (32 rows x 64 columns) an epilogue warp handles, in order: tile `first + i * stride`
+// (while below `count`), columns 64 c .. of it, c = 0 .. ppt - 1.
+struct XWalk {
+  int first, stride, count, num_n;
+  int tile_rows, row_off;  // rows per tile step; this warp's row offset inside the tile
+  int bn, ppt;             // tile width; pieces per tile = bn / 64
+};
+// Coordinates of piece p; false if there is no such piece or it lies outside the M x N matrix.
+__device__ __forceinline__ bool piece_xy(const XWalk& w, uint32_t p, long M, int N, int& x, int& y) {
+  const long t = (long)w.first + (long)(p / (uint32_t)w.ppt) * w.stride;
+  if (t >= w.count) return false;
+  x = (int)(t % w.num_n) * w.bn + (int)(p % (uint32_t)w.ppt) * 64;
+  y = (int)(t / w.num_n) * w.tile_rows + w.row_off;
+  return x < N && y < M;
+}
+// One lane: fetch the old x_hi / x_lo values of piece p into its staging set.
+__device__ __forceinline__ void x_fetch(const XWalk& w, uint32_t p, long M, int N, const CUtensorMap* t_hi,
+                                        const CUtensorMap* t_lo, uint32_t stage_base, uint32_t xbar0, uint32_t& armed) {
+  int x, y;
+  if (!piece_xy(w, p, M, N, x, y)) return;
+  const uint32_t set = p % kXSets;
+  // The set was last used by piece p - kXSets.  This runs while piece p - kXLook is current, after
+  // the groups of all earlier pieces were committed: at most kXSets - kXLook - 1 of them may still
+  // be reading shared memory.
+  bulk_wait_read<kXSets - kXLook - 1>();
+  mbar_arrive_expect_tx(xbar0 + 8u * set, 8192);
+  tma_load_2d(stage_base + set * 8192u, t_hi, x, y, xbar0 + 8u * set);
+  tma_load_2d(stage_base + set * 8192u + 4096u, t_lo, x, y, xbar0 + 8u * set);
+  armed |= 1u << set;
+}
+struct XState {
+  uint32_t piece;   // pieces handled so far
+  uint32_t phase;   // bit s: parity of staging set s's barrier to wait for next
+  uint32_t armed;   // lane 0: sets with a fetch in flight
+};
+// One tile: x <- x + acc + bias in place in shared memory, pieces stored back by TMA, the row's
+// (sum, sum of squares) over each 128 columns written to stats_out.  False after a timed-out wait.
+template <int BN>
+__device__ __forceinline__ bool epilogue_tile_split(const EpiParams& ep, const CUtensorMap* t_hi, const CUtensorMap* t_lo,
+                                                    uint32_t t_row, int m0, int n0, long M, int N, int quarter, int lane,
+                                                    uint32_t stage_base, uint32_t xbar0, const XWalk& w, XState& st,
+                                                    volatile int* abort_flag) {
+  const long row = (long)m0 + quarter * 32 + lane;
+  float s1 = 0.f, s2 = 0.f;
+#pragma unroll 1
+  for (int c = 0; c < BN / 64; ++c) {
+    const uint32_t p = st.piece;
+    if (lane == 0) x_fetch(w, p + kXLook, M, N, t_hi, t_lo, stage_base, xbar0, st.armed);
+    const bool valid = n0 + c * 64 < N && (long)m0 + quarter * 32 < M;
+    if (valid) {
+      const uint32_t set = p % kXSets;
+      const uint32_t buf = stage_base + set * 8192u;
+      bool ok = mbar_wait(xbar0 + 8u * set, (st.phase >> set) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return false;
+      st.phase ^= 1u << set;
+      st.armed &= ~(1u << set);
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t a32[32];
+        float v[32];
+        tmem_ld_32x32(t_row + c * 64 + hf * 32, a32);
+        tmem_ld_wait();
+        bias_act32<kEpiResidSplit>(ep, n0 + c * 64 + hf * 32, N, a32, v, make_float2(0.f, 0.f));
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t a = buf + lane * 128 + (((hf * 4 + j) ^ (lane & 7)) << 4);
+          uint32_t h[4], l[4];
+          ld_shared_v4(a, h[0], h[1], h[2], h[3]);
+          ld_shared_v4(a + 4096u, l[0], l[1], l[2], l[3]);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            // hi + lo is exact in float32 (16 significant bits)
+            const float x0 = (__uint_as_float(h[q] << 16) + __uint_as_float(l[q] << 16)) + v[8 * j + 2 * q];
+            const float x1 = (__uint_as_float(h[q] & 0xffff0000u) + __uint_as_float(l[q] & 0xffff0000u)) + v[8 * j + 2 * q + 1];
+            s1 += x0 + x1;
+            s2 = fmaf(x0, x0, fmaf(x1, x1, s2));
+            split_bf16x2(x0, x1, h[q], l[q]);
+          }
+          st_shared_v4(a, h[0], h[1], h[2], h[3]);
+          st_shared_v4(a + 4096u, l[0], l[1], l[2], l[3]);
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        tma_store_2d(t_hi, buf, n0 + c * 64, m0 + quarter * 32);
+        tma_store_2d(t_lo, buf + 4096u, n0 + c * 64, m0 + quarter * 32);
+      }
+    }
+    if (lane == 0) bulk_commit();  // one group per piece, empty for a piece outside the matrix (x_fetch counts groups)
+    ++st.piece;
+    if (c & 1) {  // 128 columns done
+      if (valid && row < M) ep.stats_out[(long)((n0 + c * 64) >> 7) * ep.stats_pitch + row] = make_float2(s1, s2);
+      s1 = s2 = 0.f;
+    }
+  }
+  return true;
+}
+// After a timed-out wait: let the fetches this lane issued land before the CTA's shared memory is released.
+__device__ __forceinline__ void x_drain(uint32_t xbar0, const XState& st) {
+  for (uint32_t s = 0; s < (uint32_t)kXSets; ++s) {
+    if (!(st.armed & (1u << s))) continue;
+    for (uint32_t it = 0; it < (1u << 20); ++it)
+      if (mbar_try_wait(xbar0 + 8u * s, (st.phase >> s) & 1u)) break;
+  }
+}
+
+// Bounded wait (after a timed-out wait elsewhere in the CTA) for the operand copies a producer
+// thread has in flight: bit s of `armed` = stage s has a copy whose barrier phase has parity bit s
+// of `parity`.
+__device__ __forceinline__ void drain_stages(uint32_t full_bar0, int stages, uint32_t armed, uint32_t parity) {
+  for (int s = 0; s < stages; ++s) {
+    if (!(armed & (1u << s))) continue;
+    for (uint32_t it = 0; it < (1u << 20); ++it)
+      if (mbar_try_wait(full_bar0 + 8u * s, (parity >> s) & 1u)) break;
+  }
+}
+
+// Single-CTA kernel, 128 x 128 tiles: the small-M regime, where 256 x 256 tiles would leave most
+// CTA pairs idle.  tmap_c is the bf16 output map, or x_hi's (with tmap_c2 = x_lo's) for kEpiResidSplit.
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
     const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-    const __grid_constant__ CUtensorMap tmap_c, long M, int N, int K, int a_cols, EpiParams ep, int* err_flag) {
-  using Cfg = GemmCfg<BN>;
+    const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_c2, long M, int N, int K,
+    int a_cols, EpiParams ep, int* err_flag) {
+  using Cfg = SmemPlan<BN, EPI>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -174,10 +344,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
   auto empty_bar = [&](int s) { return bar_base + 8u * (Cfg::kStages + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * Cfg::kStages + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * Cfg::kStages + 2 + a); };
-  volatile uint32_t* tmem_slot =
-      reinterpret_cast<volatile uint32_t*>(smem_gen + Cfg::kBarOffset + 8 * (2 * Cfg::kStages + 4));
-  volatile int* abort_flag =
-      reinterpret_cast<volatile int*>(smem_gen + Cfg::kBarOffset + 8 * (2 * Cfg::kStages + 4) + 8);
+  const uint32_t xbar_base = bar_base + 8u * (2 * Cfg::kStages + 4);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + Cfg::kBarOffset + 8 * Cfg::kNumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + Cfg::kBarOffset + 8 * Cfg::kNumBars + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -190,11 +359,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
       mbar_init(tfull_bar(a), 1);
       mbar_init(tempty_bar(a), 4);
     }
+    for (int i = 0; i < 4 * kXSets; ++i) mbar_init(xbar_base + 8u * i, 1);
     *abort_flag = 0;
     fence_mbar_init();
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::kTmemCols);
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 2 * BN);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -235,12 +405,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
       }
       if (!ok) {
         atomicExch(err_flag, 1);
-        // Let the copies this thread issued land before the CTA's shared memory is released.
-        for (int s = 0; s < Cfg::kStages; ++s) {
-          if (!(armed & (1u << s))) continue;
-          for (uint32_t it = 0; it < (1u << 20); ++it)
-            if (mbar_try_wait(full_bar(s), (armed_parity >> s) & 1u)) break;
-        }
+        drain_stages(full_bar(0), Cfg::kStages, armed, armed_parity);
       }
     }
   } else if (warp == 1) {
@@ -277,7 +442,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
     }
   } else {
     const int quarter = warp & 3;  // TMEM lanes this warp may read: 32 * quarter .. + 31
-    const uint32_t stage_base = smem_base + Cfg::kStagingOffset + (uint32_t)((warp - 2) * 8192);
+    const uint32_t stage_base = smem_base + Cfg::kStagingOffset + (uint32_t)((warp - 2) * Cfg::kStagingPerWarp);
+    const uint32_t xbar0 = xbar_base + 8u * (uint32_t)((warp - 2) * kXSets);
+    const XWalk walk{(int)blockIdx.x, (int)gridDim.x, num_tiles, num_n, kBM, quarter * 32, BN, BN / 64};
+    XState xs{0u, 0u, 0u};
+    if (EPI == kEpiResidSplit && lane == 0) {
+      prefetch_tmap(&tmap_c);
+      prefetch_tmap(&tmap_c2);
+      for (uint32_t p = 0; p < (uint32_t)kXLook; ++p) x_fetch(walk, p, M, N, &tmap_c, &tmap_c2, stage_base, xbar0, xs.armed);
+    }
     uint32_t piece = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -285,42 +458,36 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
       const int m0 = (tile / num_n) * kBM, n0 = (tile % num_n) * BN;
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        tc_fence_after();
+        const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+        if constexpr (EPI == kEpiResidSplit)
+          ok = epilogue_tile_split<BN>(ep, &tmap_c, &tmap_c2, t_row, m0, n0, M, N, quarter, lane, stage_base, xbar0, walk, xs,
+                                       abort_flag);
+        else
+          epilogue_tile<BN, EPI>(ep, &tmap_c, t_row, m0, n0, M, N, K, quarter, lane, stage_base, piece);
+      }
       if (!ok) {
-        if (lane == 0) atomicExch(err_flag, 3);
+        if (lane == 0) {
+          atomicExch(err_flag, 3);
+          x_drain(xbar0, xs);
+        }
         break;
       }
-      tc_fence_after();
-      epilogue_tile<BN, EPI>(ep, &tmap_c, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN), m0, n0,
-                             M, N, quarter, lane, stage_base, piece);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
-    if (lane == 0) bulk_wait_all();  // every store / reduction this lane issued has completed
+    if (lane == 0) bulk_wait_all();  // every store this lane issued has completed
   }
 
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    tmem_dealloc(tmem_base, 2 * BN);
   }
-}
-
-// Work units of the CTA-pair kernel.  Tiles are dealt round-robin to the pairs; the tiles of the
-// last, partial round are cut along K into `split` parts (only for the residual epilogue, whose
-// float32 add-reduction makes partial sums free to combine), so that every pair has work in
-// that round too.  Unit u < full is the whole tile u; the others are (tile, K part) pairs, with
-// the bias added by part 0 alone.
-struct GemmUnit {
-  int tile, kb0, kb1;
-  bool first;
-};
-__device__ __forceinline__ GemmUnit gemm_unit(int u, int full, int rem, int split, int num_k) {
-  if (u < full) return GemmUnit{u, 0, num_k, true};
-  const int v = u - full, part = v / rem;
-  return GemmUnit{full + v % rem, part * num_k / split, (part + 1) * num_k / split, part == 0};
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -331,33 +498,28 @@ __device__ __forceinline__ GemmUnit gemm_unit(int u, int full, int rem, int spli
 //     of the pair's first CTA (the leader), which alone issues the MMAs;
 //   - tcgen05.commit multicasts "stage free" and "accumulator ready" to both CTAs;
 //   - the epilogue warps of both CTAs arrive on the leader's "accumulator drained" barrier.
+// Tiles are dealt round-robin to the pairs.
 template <int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
     const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-    const __grid_constant__ CUtensorMap tmap_c, long M, int N, int K, int a_cols, EpiParams ep, int* err_flag,
-    int tail_split) {
+    const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_c2, long M, int N, int K,
+    int a_cols, EpiParams ep, int* err_flag) {
   constexpr int BN = 256;
-  // The float32 add-reduction holds its staging buffer for ~2 us (the L2 performs the additions), so
-  // with two buffers per warp the residual epilogue is latency-bound at ~13 GB/s per CTA and the
-  // K = 1280 out-projection waits for it: that epilogue gets four buffers per warp, paid for with
-  // one operand stage.
-  constexpr int kStages = EPI == kEpiBiasResid ? 5 : 6;
-  constexpr int kBufs = EPI == kEpiBiasResid ? 4 : 2;
-  constexpr int kABytes = kBM * kBK * 2;          // this CTA's 128 rows of A
-  constexpr int kBBytes = (BN / 2) * kBK * 2;     // this CTA's 128 of the 256 W rows
-  constexpr int kStageBytes = kABytes + kBBytes;  // 32 KB
-  constexpr int kStagingOffset = kStages * kStageBytes;
-  constexpr int kBarOffset = kStagingOffset + 4 * kBufs * 4096;
+  using Cfg = SmemPlan<BN / 2, EPI>;  // this CTA's 128 rows of A and 128 of the 256 W rows per stage: 32 KB
+  constexpr int kStages = Cfg::kStages;
+  constexpr int kABytes = Cfg::kABytes;
+  constexpr int kStageBytes = Cfg::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_base = smem_base + kBarOffset;
+  const uint32_t bar_base = smem_base + Cfg::kBarOffset;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + kBarOffset + 8 * (2 * kStages + 4));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + kBarOffset + 8 * (2 * kStages + 4) + 8);
+  const uint32_t xbar_base = bar_base + 8u * (2 * kStages + 4);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + Cfg::kBarOffset + 8 * Cfg::kNumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + Cfg::kBarOffset + 8 * Cfg::kNumBars + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();  // 0 = leader
@@ -372,6 +534,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
       mbar_init(tfull_bar(a), 1);   // one multicast commit
       mbar_init(tempty_bar(a), 8);  // used in the leader only: 4 epilogue warps of each CTA
     }
+    for (int i = 0; i < 4 * kXSets; ++i) mbar_init(xbar_base + 8u * i, 1);
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -390,8 +553,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
   const int num_n = (N + BN - 1) / BN;
   const int num_k = (K + kBK - 1) / kBK;
   const int num_tiles = num_m * num_n;
-  const int full_tiles = (num_tiles / n_pairs) * n_pairs, rem_tiles = num_tiles - full_tiles;
-  const int num_units = full_tiles + rem_tiles * tail_split;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -400,11 +561,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int u = pair_id; ok && u < num_units; u += n_pairs) {
-        const GemmUnit w = gemm_unit(u, full_tiles, rem_tiles, tail_split, num_k);
-        const int m0 = (w.tile / num_n) * (2 * kBM) + (int)rank * kBM;
-        const int n0 = (w.tile % num_n) * BN + (int)rank * (BN / 2);
-        for (int kb = w.kb0; kb < w.kb1; ++kb) {
+      for (int tile = pair_id; ok && tile < num_tiles; tile += n_pairs) {
+        const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
+        const int n0 = (tile % num_n) * BN + (int)rank * (BN / 2);
+        for (int kb = 0; kb < num_k; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t leader_full = map_to_cta(full_bar(stage), 0);  // the leader CTA's barrier
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * kStageBytes);
@@ -415,7 +575,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) atomicExch(err_flag, 4);
+      if (!ok) {
+        atomicExch(err_flag, 4);
+        // This thread's copies signal the leader's barriers, which only the leader's MMA thread
+        // follows; what can be waited for here is that the stages it filled were consumed, i.e. one
+        // more lap of the "stage free" barriers, each wait bounded.
+        for (int s = 0; s < kStages; ++s)
+          for (uint32_t it = 0; it < (1u << 16); ++it)
+            if (mbar_try_wait(empty_bar(s), (s < stage ? phase : phase ^ 1u))) break;
+      }
     }
   } else if (warp == 1) {
     if (rank == 0 && lane == 0) {
@@ -425,12 +593,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int u = pair_id; ok && u < num_units; u += n_pairs) {
-        const GemmUnit w = gemm_unit(u, full_tiles, rem_tiles, tail_split, num_k);
+      for (int tile = pair_id; ok && tile < num_tiles; tile += n_pairs) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = w.kb0; kb < w.kb1; ++kb) {
+        for (int kb = 0; kb < num_k; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * kStageBytes;
@@ -438,7 +605,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
           const uint64_t bdesc = umma_desc_k_sw128(sa + kABytes);
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k)
-            umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > w.kb0 || k != 0) ? 1u : 0u);
+            umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
           umma_commit_pair(empty_bar(stage), 3);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -450,23 +617,39 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_pair_kernel(
     }
   } else {
     const int quarter = warp & 3;
-    const uint32_t stage_base = smem_base + kStagingOffset + (uint32_t)((warp - 2) * kBufs * 4096);
+    const uint32_t stage_base = smem_base + Cfg::kStagingOffset + (uint32_t)((warp - 2) * Cfg::kStagingPerWarp);
+    const uint32_t xbar0 = xbar_base + 8u * (uint32_t)((warp - 2) * kXSets);
+    const XWalk walk{pair_id, n_pairs, num_tiles, num_n, 2 * kBM, (int)rank * kBM + quarter * 32, BN, BN / 64};
+    XState xs{0u, 0u, 0u};
+    if (EPI == kEpiResidSplit && lane == 0) {
+      prefetch_tmap(&tmap_c);
+      prefetch_tmap(&tmap_c2);
+      for (uint32_t p = 0; p < (uint32_t)kXLook; ++p) x_fetch(walk, p, M, N, &tmap_c, &tmap_c2, stage_base, xbar0, xs.armed);
+    }
     uint32_t piece = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (int u = pair_id; u < num_units; u += n_pairs) {
-      const GemmUnit w = gemm_unit(u, full_tiles, rem_tiles, tail_split, num_k);
-      const int m0 = (w.tile / num_n) * (2 * kBM) + (int)rank * kBM;
-      const int n0 = (w.tile % num_n) * BN;
+    for (int tile = pair_id; tile < num_tiles; tile += n_pairs) {
+      const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
+      const int n0 = (tile % num_n) * BN;
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        tc_fence_after();
+        const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+        if constexpr (EPI == kEpiResidSplit)
+          ok = epilogue_tile_split<BN>(ep, &tmap_c, &tmap_c2, t_row, m0, n0, M, N, quarter, lane, stage_base, xbar0, walk, xs,
+                                       abort_flag);
+        else
+          epilogue_tile<BN, EPI>(ep, &tmap_c, t_row, m0, n0, M, N, K, quarter, lane, stage_base, piece);
+      }
       if (!ok) {
-        if (lane == 0) atomicExch(err_flag, 6);
+        if (lane == 0) {
+          atomicExch(err_flag, 6);
+          x_drain(xbar0, xs);
+        }
         break;
       }
-      tc_fence_after();
-      epilogue_tile<BN, EPI, kBufs>(ep, &tmap_c, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN), m0, n0,
-                             M, N, quarter, lane, stage_base, piece, w.first);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
@@ -521,118 +704,95 @@ bool make_tmap_out(const TmaApi& api, CUtensorMap* m, const void* base, int elem
   return make_tmap_2d(api, m, base, elem_bytes, cols, rows, cols, elem_bytes == 2 ? 64 : 32, 32);
 }
 
-template <int BN, int EPI>
+template <int EPI>
 static cudaError_t configure_one() {
-  return cudaFuncSetAttribute(gemm_bf16_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              GemmCfg<BN>::kSmemBytes);
+  return cudaFuncSetAttribute(gemm_bf16_kernel<128, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              SmemPlan<128, EPI>::kSmemBytes);
 }
-
-constexpr int kPairSmemBytes = 6 * 32768 + 4 * 2 * 4096 + 256 + 1024;
 
 template <int EPI>
 static cudaError_t configure_pair() {
   cudaError_t e = cudaFuncSetAttribute(gemm_bf16_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kPairSmemBytes);
+                                       SmemPlan<128, EPI>::kSmemBytes);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(gemm_bf16_pair_kernel<EPI>, cudaFuncAttributeNonPortableClusterSizeAllowed, 0);
 }
 
+// Function attributes are per device: called by every create, on the device that is current then.
 cudaError_t gemm_bf16_configure() {
   cudaError_t e;
   if ((e = configure_pair<kEpiBias>()) != cudaSuccess) return e;
   if ((e = configure_pair<kEpiBiasGelu>()) != cudaSuccess) return e;
-  if ((e = configure_pair<kEpiBiasResid>()) != cudaSuccess) return e;
   if ((e = configure_pair<kEpiConv1>()) != cudaSuccess) return e;
   if ((e = configure_pair<kEpiConv2>()) != cudaSuccess) return e;
-  if ((e = configure_one<256, kEpiBias>()) != cudaSuccess) return e;
-  if ((e = configure_one<256, kEpiBiasGelu>()) != cudaSuccess) return e;
-  if ((e = configure_one<256, kEpiBiasResid>()) != cudaSuccess) return e;
-  if ((e = configure_one<256, kEpiConv1>()) != cudaSuccess) return e;
-  if ((e = configure_one<256, kEpiConv2>()) != cudaSuccess) return e;
-  if ((e = configure_one<128, kEpiBias>()) != cudaSuccess) return e;
-  if ((e = configure_one<128, kEpiBiasGelu>()) != cudaSuccess) return e;
-  if ((e = configure_one<128, kEpiBiasResid>()) != cudaSuccess) return e;
+  if ((e = configure_pair<kEpiLnBias>()) != cudaSuccess) return e;
+  if ((e = configure_pair<kEpiLnBiasGelu>()) != cudaSuccess) return e;
+  if ((e = configure_pair<kEpiResidSplit>()) != cudaSuccess) return e;
+  if ((e = configure_one<kEpiBias>()) != cudaSuccess) return e;
+  if ((e = configure_one<kEpiBiasGelu>()) != cudaSuccess) return e;
+  if ((e = configure_one<kEpiLnBias>()) != cudaSuccess) return e;
+  if ((e = configure_one<kEpiLnBiasGelu>()) != cudaSuccess) return e;
+  if ((e = configure_one<kEpiResidSplit>()) != cudaSuccess) return e;
   return cudaSuccess;
 }
 
-template <int BN, int EPI>
-static void launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
-                       int a_cols, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
-  const long tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
+template <int EPI>
+static void launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
+                       long M, int N, int K, int a_cols, const EpiParams& ep, int* err_flag, int num_sms, bool pdl,
+                       cudaStream_t s) {
+  const long tiles = ((M + kBM - 1) / kBM) * ((N + 127) / 128);
   const int grid = (int)(tiles < num_sms ? tiles : num_sms);
-  launch_dependent(gemm_bf16_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), GemmCfg<BN>::kSmemBytes, s, 1, ta, tb, tc,
-                   M, N, K, a_cols, ep, err_flag);
+  launch_dependent(gemm_bf16_kernel<128, EPI>, dim3(grid), dim3(kGemmThreads), SmemPlan<128, EPI>::kSmemBytes, s, 1, pdl,
+                   ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag);
 }
-
-// pair = 1: CTA-pair kernel (W maps must then use 128-row boxes); 0: single-CTA kernel
-static int g_gemm_use_pair = 1;
-static int g_gemm_tail_split = 0;
-static int g_gemm_small_tiles = 1;
-void gemm_bf16_set_pair(int on) { g_gemm_use_pair = on; }
-int gemm_bf16_uses_pair() { return g_gemm_use_pair; }
-void gemm_bf16_set_tail_split(int on) { g_gemm_tail_split = on; }
-void gemm_bf16_set_small_tiles(int on) { g_gemm_small_tiles = on; }
 
 template <int EPI>
-static void launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
-                        int a_cols, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
+static void launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
+                        long M, int N, int K, int a_cols, const EpiParams& ep, int* err_flag, int num_sms, bool pdl,
+                        cudaStream_t s) {
   const long tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + 255) / 256);
   const long max_pairs = num_sms / 2;
-  long pairs = tiles < max_pairs ? tiles : max_pairs;
-  // the residual epilogue lets the tiles of the last, partial round be cut along K (see GemmUnit);
-  // with fewer tiles than pairs that round is the only one, and more pairs are launched for it
-  int tail_split = 1;
-  if (EPI == kEpiBiasResid && g_gemm_tail_split) {
-    const long num_k = (K + kBK - 1) / kBK;
-    if (tiles < max_pairs) pairs = std::min(max_pairs, tiles * num_k);
-    const long rem = tiles % pairs;
-    if (rem > 0) tail_split = (int)std::max(1L, std::min(pairs / rem, num_k));
-    if (tiles < max_pairs) pairs = tiles * tail_split;
-  }
-  launch_dependent(gemm_bf16_pair_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(kGemmThreads), kPairSmemBytes, s, 2,
-                   ta, tb, tc, M, N, K, a_cols, ep, err_flag, tail_split);
+  const long pairs = tiles < max_pairs ? tiles : max_pairs;
+  launch_dependent(gemm_bf16_pair_kernel<EPI>, dim3((unsigned)(2 * pairs)), dim3(kGemmThreads),
+                   SmemPlan<128, EPI>::kSmemBytes, s, 2, pdl, ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag);
 }
 
-void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
-                      int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s) {
+void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
+                      long M, int N, int K, int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms,
+                      const LaunchOpts& opt, cudaStream_t s) {
   if (M <= 0 || N <= 0 || K <= 0) return;
-  if (g_gemm_use_pair) {
-    // Small problems leave most CTA pairs idle or waste most of a last round of 256 x 256 tiles:
-    // 128 x 128 tiles on single CTAs (same tensor maps: both use 128-row boxes) quarter the
-    // granularity.  Estimated rounds, a 128 x 128 tile counted as half a pair tile's time times
-    // kSmallTilePenalty for its lower efficiency (it reads shared memory at the full 128 B/clk;
-    // measured: a round of small tiles takes ~0.8 of a round of pair tiles).
-    if (g_gemm_small_tiles && epi <= kEpiBiasResid && a_cols == K) {
-      constexpr double kSmallTilePenalty = 1.6;
-      const long t_pair = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + 255) / 256);
-      const long t_small = ((M + kBM - 1) / kBM) * ((N + 127) / 128);
-      const long n_pairs = num_sms / 2;
-      const double r_pair = (double)((t_pair + n_pairs - 1) / n_pairs);
-      const double r_small = (double)((t_small + num_sms - 1) / num_sms) * 0.5 * kSmallTilePenalty;
-      if (r_small < r_pair) {
-        switch (epi) {
-          case kEpiBias: launch_one<128, kEpiBias>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-          case kEpiBiasGelu: launch_one<128, kEpiBiasGelu>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-          default: launch_one<128, kEpiBiasResid>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-        }
-        return;
+  const bool pdl = opt.pdl != 0;
+  // Small problems leave most CTA pairs idle or waste most of a last round of 256 x 256 tiles:
+  // 128 x 128 tiles on single CTAs (same tensor maps: both use 128-row boxes) quarter the
+  // granularity.  Estimated rounds, a 128 x 128 tile counted as half a pair tile's time times
+  // kSmallTilePenalty for its lower efficiency (it reads shared memory at the full 128 B/clk;
+  // measured: a round of small tiles takes ~0.8 of a round of pair tiles).
+  if (opt.small_tiles && epi != kEpiConv1 && epi != kEpiConv2 && a_cols == K) {
+    constexpr double kSmallTilePenalty = 1.6;
+    const long t_pair = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + 255) / 256);
+    const long t_small = ((M + kBM - 1) / kBM) * ((N + 127) / 128);
+    const long n_pairs = num_sms / 2;
+    const double r_pair = (double)((t_pair + n_pairs - 1) / n_pairs);
+    const double r_small = (double)((t_small + num_sms - 1) / num_sms) * 0.5 * kSmallTilePenalty;
+    if (r_small < r_pair) {
+      switch (epi) {
+        case kEpiBias: launch_one<kEpiBias>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+        case kEpiBiasGelu: launch_one<kEpiBiasGelu>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+        case kEpiLnBias: launch_one<kEpiLnBias>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+        case kEpiLnBiasGelu: launch_one<kEpiLnBiasGelu>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+        default: launch_one<kEpiResidSplit>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
       }
+      return;
     }
-    switch (epi) {
-      case kEpiBias: launch_pair<kEpiBias>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-      case kEpiBiasGelu: launch_pair<kEpiBiasGelu>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-      case kEpiBiasResid: launch_pair<kEpiBiasResid>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-      case kEpiConv1: launch_pair<kEpiConv1>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-      default: launch_pair<kEpiConv2>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-    }
-    return;
   }
   switch (epi) {
-    case kEpiBias: launch_one<256, kEpiBias>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-    case kEpiBiasGelu: launch_one<256, kEpiBiasGelu>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-    case kEpiBiasResid: launch_one<256, kEpiBiasResid>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-    case kEpiConv1: launch_one<256, kEpiConv1>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
-    default: launch_one<256, kEpiConv2>(ta, tb, tc, M, N, K, a_cols, ep, err_flag, num_sms, s); break;
+    case kEpiBias: launch_pair<kEpiBias>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+    case kEpiBiasGelu: launch_pair<kEpiBiasGelu>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+    case kEpiConv1: launch_pair<kEpiConv1>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+    case kEpiConv2: launch_pair<kEpiConv2>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+    case kEpiLnBias: launch_pair<kEpiLnBias>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+    case kEpiLnBiasGelu: launch_pair<kEpiLnBiasGelu>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+    default: launch_pair<kEpiResidSplit>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
   }
 }
 

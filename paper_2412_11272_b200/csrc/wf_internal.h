@@ -26,7 +26,17 @@ enum Epilogue : int {
   kEpiBiasGelu = 1,   // out = gelu(acc + bias)
   kEpiBiasResid = 2,  // resid(f32) += acc + bias
   kEpiConv1 = 3,      // out[row] = row_valid[row] ? gelu(acc + bias) : 0
-  kEpiConv2 = 4       // resid(f32)[dst[row]] = gelu(acc + bias) + pe[pos[row]] (dst < 0: skip)
+  kEpiConv2 = 4,      // x[dst[row]] = gelu(acc + bias) + pe[pos[row]] (dst < 0: skip); x is f32 on the
+                      // float32 path, the split bf16 residual stream (+ row statistics) on the bf16 path
+  // bf16 path only.  The residual stream x is held as two bf16 planes, x = x_hi + x_lo with
+  // x_hi = bf16(x) and x_lo = bf16(x - x_hi) (16 significant bits), so that x_hi is at once the
+  // A operand of the GEMM that follows a LayerNorm.  That LayerNorm is folded into the GEMM:
+  // with W' = W diag(gamma) (rounded to bf16), s[n] = sum_k W'[n,k], c[n] = bias[n] + sum_k W[n,k] beta[k],
+  //   LN(x) W^T + bias = rstd (x W'^T - mean s) + c,
+  // mean and rstd coming from per-row partial sums that the producer of x leaves behind.
+  kEpiLnBias = 5,      // out = rstd (acc - mean s) + c
+  kEpiLnBiasGelu = 6,  // out = gelu(rstd (acc - mean s) + c)
+  kEpiResidSplit = 7   // (x_hi, x_lo) <- split(x_hi + x_lo + acc + bias); row statistics written
 };
 
 struct EpiParams {
@@ -37,6 +47,19 @@ struct EpiParams {
   const int* row_valid;  // kEpiConv1: one int per GEMM row
   const int2* row_dst;   // kEpiConv2: (destination token row or -1, position in sequence)
   const float* pe;       // kEpiConv2: sinusoid table [n_ctx, N]
+  // bf16 path, LayerNorm folded into the consumer / statistics left by the producer:
+  const float* colsum;      // kEpiLn*: s[n]; `bias` then holds c[n]
+  const float2* stats_in;   // kEpiLn*: [K / 128][stats_pitch] partial (sum, sum of squares) of 128 columns of x
+  float2* stats_out;        // kEpiResidSplit, kEpiConv2 (bf16): the same layout over the N output columns
+  long stats_pitch;         // rows per partial plane
+  __nv_bfloat16* x_hi;      // kEpiConv2 (bf16): planes of the residual stream, row pitch ldc
+  __nv_bfloat16* x_lo;
+};
+
+// Per-handle launch options of the bf16 path.
+struct LaunchOpts {
+  int pdl;          // launch with programmatic stream serialization (a kernel's set-up overlaps its predecessor's tail)
+  int small_tiles;  // GEMMs too small to fill the CTA pairs run 128 x 128 tiles on single CTAs
 };
 
 // Offsets (in ints) of the per-call metadata arrays inside one device int buffer.
@@ -58,12 +81,10 @@ struct MetaLayout {
 // ---- kernel launch with optional cluster size and programmatic stream serialization.
 // With the latter the kernel may begin (set up barriers, allocate tensor memory) while the kernel
 // before it in the stream drains; it must call ptx::griddep_wait() before it touches global
-// memory.  pdl_enabled() is process-wide (wf_api.cu; on unless WF_PDL=0 in the environment).
-int pdl_enabled();
-void pdl_set(int on);
+// memory.
 template <typename... P, typename... A>
 inline cudaError_t launch_dependent(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
-                                    int cluster_x, A&&... args) {
+                                    int cluster_x, bool pdl, A&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -78,7 +99,7 @@ inline cudaError_t launch_dependent(void (*kernel)(P...), dim3 grid, dim3 block,
     attrs[n].val.clusterDim.z = 1;
     ++n;
   }
-  if (pdl_enabled()) {
+  if (pdl) {
     attrs[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attrs[n].val.programmaticStreamSerializationAllowed = 1;
     ++n;
@@ -96,6 +117,7 @@ void launch_build_tables(float* dft_basis /*[2][kFold][kBasisCols]*/, float* pe,
 // mel_fb_t holds the transposed filterbank [201][n_mel] followed by n_mel int2 (launch_mel_bin_ranges):
 // per channel, the run of bins [first, last + 1) that holds its non-zero weights.
 void launch_mel_bin_ranges(float* mel_fb_t, int n_mel, cudaStream_t s);
+cudaError_t frontend_configure();
 void launch_frontend(const float* audio, const int* meta, MetaLayout ml, int B, int n_tiles,
                      const float* dft_basis, const float* mel_fb_t /*[201][n_mel]*/, int n_mel,
                      float* logmel /*[sum T, n_mel]*/, int* seq_max /*[B] ordered ints*/,
@@ -123,8 +145,7 @@ void launch_stream_max(const float* logmel, const int* meta, MetaLayout ml, int 
 // ---- SIMT float32 kernels and element-wise kernels (wf_simt.cu)
 void launch_gemm_f32(const float* A, long lda, const float* W, long ldw, long M, int N, int K,
                      int epi, const EpiParams& ep, cudaStream_t s);
-void launch_layernorm(const float* x, const float* g, const float* b, void* out, int out_bf16,
-                      long M, int d, cudaStream_t s);
+void launch_layernorm(const float* x, const float* g, const float* b, float* out, long M, int d, cudaStream_t s);
 void launch_attention_f32(const float* qkv, float* out, const int* meta, MetaLayout ml, int n_work,
                           int d_model, cudaStream_t s);
 void launch_convert(const float* src, void* dst, long n, int dst_bf16, cudaStream_t s);
@@ -145,21 +166,24 @@ bool make_tmap_bf16(const TmaApi& api, CUtensorMap* m, const void* base, uint64_
 bool make_tmap_out(const TmaApi& api, CUtensorMap* m, const void* base, int elem_bytes, uint64_t cols,
                    uint64_t rows);
 cudaError_t gemm_bf16_configure();
-// 1 (default): CTA-pair kernel, W tensor maps need 128-row boxes; 0: single-CTA kernel, 256-row boxes
-int gemm_bf16_uses_pair();
-void gemm_bf16_set_pair(int on);
-// 1: residual-epilogue GEMMs cut the tiles of their last, partial round along K (default 0:
-// the order of the float32 residual additions, and with it every output bit, is then fixed)
-void gemm_bf16_set_tail_split(int on);
-// 1 (default): GEMMs too small to fill the CTA pairs with 256 x 256 tiles run 128 x 128 tiles on single CTAs
-void gemm_bf16_set_small_tiles(int on);
+// W tensor maps use 128-row boxes (both kernels stage 128 W rows per copy).
 // a_cols: stored row length of A in elements (K for a plain GEMM; smaller when one GEMM row
 // spans several consecutive stored rows, which must then be a multiple of 64).
-// tc: output map (bf16 out for kEpiBias/kEpiBiasGelu/kEpiConv1, float32 residual for
-// kEpiBiasResid; unused by kEpiConv2).  Rows of the output between M and the next multiple of
-// 128 are written too when the map has them: outputs must be capacity-sized or exactly M rows.
-void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, long M, int N, int K,
-                      int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms, cudaStream_t s);
+// tc: bf16 output map (kEpiBias, kEpiBiasGelu, kEpiLn*, kEpiConv1); kEpiResidSplit: tc / tc2 are the
+// maps of x_hi / x_lo (make_tmap_out, used for the fetch and for the store); unused by kEpiConv2.
+// Rows of the output between M and the next multiple of 128 are written too when the map has
+// them: outputs must be capacity-sized or exactly M rows.
+void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
+                      long M, int N, int K, int a_cols, int epi, const EpiParams& ep, int* err_flag, int num_sms,
+                      const LaunchOpts& opt, cudaStream_t s);
+// Folds a LayerNorm's affine part into the weight that follows it (rows [0, N) of W [N, K] float32):
+// wg = bf16(W diag(g)), colsum[n] = sum_k float(wg[n,k]), cbias[n] = bias[n] + sum_k W[n,k] b[k]
+// (bias may be NULL = zeros).
+void launch_ln_fold(const float* W, const float* g, const float* b, const float* bias, __nv_bfloat16* wg,
+                    float* colsum, float* cbias, int N, int K, cudaStream_t s);
+// Final LayerNorm of the bf16 path: reads the split residual stream.
+void launch_layernorm_split(const __nv_bfloat16* x_hi, const __nv_bfloat16* x_lo, const float* g, const float* b,
+                            __nv_bfloat16* out, long M, int d, bool pdl, cudaStream_t s);
 
 // ---- bf16 attention on tcgen05 (wf_attention_tc.cu).  The work list at ml.attn_work holds
 // n_entries triples (sequence, first query row | kind << 30, first item): kind 0 = 256 consecutive
@@ -170,7 +194,7 @@ cudaError_t attention_bf16_configure();
 // (make_tmap_bf16 with box_rows 128 and 96)
 void launch_attention_bf16(const CUtensorMap& tmap_q, const CUtensorMap& tmap_kv, __nv_bfloat16* out,
                            const int* meta, MetaLayout ml, int n_entries, int n_items, int d_model, int* err_flag,
-                           int num_sms, cudaStream_t s);
+                           int num_sms, bool pdl, cudaStream_t s);
 
 // ---- dynamic time warping (wf_dtw.cu); meta holds 4 ints per problem:
 // cost offset in cells, tokens, frames, offset into token_start

@@ -73,8 +73,10 @@ void launch_gemm_f32(const float* A, long lda, const float* W, long ldw, long M,
 // ---------------------------------------------------------------------------------------------
 // LayerNorm over d = 128 NV channels, one warp per row, the row held in registers
 // (mean, then centred sum of squares: no cancellation), biased variance, eps 1e-5.
-template <int NV, typename OutT>
-__global__ void __launch_bounds__(256) layernorm_kernel(const float* __restrict__ x,
+// SPLIT: the row is read from the two bf16 planes of the bf16 path's residual stream (x = hi + lo).
+template <int NV, bool SPLIT, typename OutT>
+__global__ void __launch_bounds__(256) layernorm_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ x_hi,
+                                                        const __nv_bfloat16* __restrict__ x_lo,
                                                         const float* __restrict__ g,
                                                         const float* __restrict__ b,
                                                         OutT* __restrict__ out, long M) {
@@ -84,12 +86,20 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const float* __restrict_
   const int lane = threadIdx.x & 31;
   if (row >= M) return;
   constexpr int d = NV * 128;
-  const float4* xr = reinterpret_cast<const float4*>(x + row * d);
   float4 v[NV];
   float sum = 0.f;
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
-    v[i] = xr[lane + 32 * i];
+    if (SPLIT) {
+      const uint2 h = *reinterpret_cast<const uint2*>(x_hi + row * d + (lane + 32 * i) * 4);
+      const uint2 l = *reinterpret_cast<const uint2*>(x_lo + row * d + (lane + 32 * i) * 4);
+      v[i].x = __uint_as_float(h.x << 16) + __uint_as_float(l.x << 16);
+      v[i].y = __uint_as_float(h.x & 0xffff0000u) + __uint_as_float(l.x & 0xffff0000u);
+      v[i].z = __uint_as_float(h.y << 16) + __uint_as_float(l.y << 16);
+      v[i].w = __uint_as_float(h.y & 0xffff0000u) + __uint_as_float(l.y & 0xffff0000u);
+    } else {
+      v[i] = reinterpret_cast<const float4*>(x + row * d)[lane + 32 * i];
+    }
     sum += (v[i].x + v[i].y) + (v[i].z + v[i].w);
   }
 #pragma unroll
@@ -118,30 +128,68 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const float* __restrict_
   }
 }
 
-template <typename OutT>
-static void layernorm_dispatch(const float* x, const float* g, const float* b, OutT* out, long M, int d,
-                               cudaStream_t s) {
+template <bool SPLIT, typename OutT>
+static void layernorm_dispatch(const float* x, const __nv_bfloat16* x_hi, const __nv_bfloat16* x_lo, const float* g,
+                               const float* b, OutT* out, long M, int d, bool pdl, cudaStream_t s) {
   unsigned grid = (unsigned)((M + 7) / 8);
+#define WF_LN_CASE(NV) \
+  case NV: launch_dependent(layernorm_kernel<NV, SPLIT, OutT>, dim3(grid), dim3(256), 0, s, 1, pdl, x, x_hi, x_lo, g, b, out, M); break;
   switch (d / 128) {
-    case 1: launch_dependent(layernorm_kernel<1, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
-    case 2: launch_dependent(layernorm_kernel<2, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
-    case 3: launch_dependent(layernorm_kernel<3, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
-    case 4: launch_dependent(layernorm_kernel<4, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
-    case 5: launch_dependent(layernorm_kernel<5, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
-    case 6: launch_dependent(layernorm_kernel<6, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
-    case 7: launch_dependent(layernorm_kernel<7, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
-    case 8: launch_dependent(layernorm_kernel<8, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
-    case 9: launch_dependent(layernorm_kernel<9, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
-    case 10: launch_dependent(layernorm_kernel<10, OutT>, dim3(grid), dim3(256), 0, s, 1, x, g, b, out, M); break;
+    WF_LN_CASE(1) WF_LN_CASE(2) WF_LN_CASE(3) WF_LN_CASE(4) WF_LN_CASE(5)
+    WF_LN_CASE(6) WF_LN_CASE(7) WF_LN_CASE(8) WF_LN_CASE(9) WF_LN_CASE(10)
     default: break;  // create() rejects d_model > 1280
   }
+#undef WF_LN_CASE
 }
 
-void launch_layernorm(const float* x, const float* g, const float* b, void* out, int out_bf16, long M,
-                      int d, cudaStream_t s) {
+void launch_layernorm(const float* x, const float* g, const float* b, float* out, long M, int d, cudaStream_t s) {
   if (M <= 0) return;
-  if (out_bf16) layernorm_dispatch<__nv_bfloat16>(x, g, b, (__nv_bfloat16*)out, M, d, s);
-  else layernorm_dispatch<float>(x, g, b, (float*)out, M, d, s);
+  layernorm_dispatch<false, float>(x, nullptr, nullptr, g, b, out, M, d, false, s);
+}
+
+void launch_layernorm_split(const __nv_bfloat16* x_hi, const __nv_bfloat16* x_lo, const float* g, const float* b,
+                            __nv_bfloat16* out, long M, int d, bool pdl, cudaStream_t s) {
+  if (M <= 0) return;
+  layernorm_dispatch<true, __nv_bfloat16>(nullptr, x_hi, x_lo, g, b, out, M, d, pdl, s);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Create-time fold of a LayerNorm's affine part into the weight that follows it; one CTA per
+// output row n: wg[n,k] = bf16(W[n,k] g[k]), colsum[n] = sum_k float(wg[n,k]) (of the rounded
+// values: the GEMM epilogue's mean * colsum then cancels the common mode of x exactly as the
+// tensor core saw it), cbias[n] = bias[n] + sum_k W[n,k] b[k].
+__global__ void __launch_bounds__(256) ln_fold_kernel(const float* __restrict__ W, const float* __restrict__ g,
+                                                      const float* __restrict__ b, const float* __restrict__ bias,
+                                                      __nv_bfloat16* __restrict__ wg, float* __restrict__ colsum,
+                                                      float* __restrict__ cbias, int K) {
+  __shared__ float red[2][8];
+  const int n = blockIdx.x, tid = threadIdx.x;
+  float s = 0.f, c = 0.f;
+  for (int k = tid; k < K; k += 256) {
+    const float w = W[(long)n * K + k];
+    const __nv_bfloat16 q = __float2bfloat16_rn(w * g[k]);
+    wg[(long)n * K + k] = q;
+    s += __bfloat162float(q);
+    c = fmaf(w, b[k], c);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, o);
+    c += __shfl_xor_sync(0xffffffffu, c, o);
+  }
+  if ((tid & 31) == 0) { red[0][tid >> 5] = s; red[1][tid >> 5] = c; }
+  __syncthreads();
+  if (tid == 0) {
+    float ts = 0.f, tc = 0.f;
+    for (int i = 0; i < 8; ++i) { ts += red[0][i]; tc += red[1][i]; }
+    colsum[n] = ts;
+    cbias[n] = tc + (bias ? bias[n] : 0.f);
+  }
+}
+void launch_ln_fold(const float* W, const float* g, const float* b, const float* bias, __nv_bfloat16* wg,
+                    float* colsum, float* cbias, int N, int K, cudaStream_t s) {
+  if (N <= 0) return;
+  ln_fold_kernel<<<N, 256, 0, s>>>(W, g, b, bias, wg, colsum, cbias, K);
 }
 
 // ---------------------------------------------------------------------------------------------

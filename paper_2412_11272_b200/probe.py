@@ -65,8 +65,19 @@ def main():
         A = torch.randn(a.M, a.K, device="cuda").to(torch.bfloat16)
         W = (torch.randn(a.N, a.K, device="cuda") / math.sqrt(a.K)).to(torch.bfloat16)
         b = torch.randn(a.N, device="cuda")
-        C = torch.zeros(a.M, a.N, device="cuda", dtype=torch.float32 if a.mode == 2 else torch.bfloat16)
-        ms = _time(lambda: enc.wf_gemm_bf16(A, W, b, a.mode, C), a.iters)
+        # --mode 0 bias, 1 bias + GELU, 2 residual update on the split stream, 3 / 4 LayerNorm folded in (4: + GELU)
+        if a.mode == 2:
+            hi = torch.randn(a.M, a.N, device="cuda").to(torch.bfloat16)
+            lo = torch.zeros_like(hi)
+            ms = _time(lambda: enc.wf_gemm_resid_bf16(A, W, b, hi, lo), a.iters)
+        elif a.mode >= 3:
+            stats = torch.stack([A.float().view(a.M, a.K // 128, 128).sum(-1).T,
+                                 (A.float() ** 2).view(a.M, a.K // 128, 128).sum(-1).T], dim=-1).contiguous()
+            cs = W.float().sum(1)
+            ms = _time(lambda: enc.wf_gemm_ln_bf16(A, stats, W, cs, b, a.mode == 4), a.iters)
+        else:
+            C = torch.zeros(a.M, a.N, device="cuda", dtype=torch.bfloat16)
+            ms = _time(lambda: enc.wf_gemm_bf16(A, W, b, a.mode, C), a.iters)
         enc.wf_check()
         out.update(M=a.M, N=a.N, K=a.K, mode=a.mode, ms=ms, tflops=2.0 * a.M * a.N * a.K / ms / 1e9)
     elif a.what == "attention":

@@ -168,7 +168,7 @@ def enc2_encode(shape, W, audio, lengths):
 
 @pytest.mark.parametrize("M,N,K", [(300, 384, 240), (1000, 1536, 512), (129, 256, 64), (4097, 1280, 1280),
                                    (77, 8, 8)])
-@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("mode", [0, 1])
 def test_tcgen05_gemm_matches_fp64(M, N, K, mode):
     shape = _small("bf16", n_layer=0)
     enc = make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000)
@@ -178,19 +178,88 @@ def test_tcgen05_gemm_matches_fp64(M, N, K, mode):
     bias = rng.normal(size=N).astype(np.float32)
     ref = A.astype(np.float64) @ Wm.astype(np.float64).T + bias
     dA, dW, db = _dev(A, torch.bfloat16), _dev(Wm, torch.bfloat16), _dev(bias)
-    if mode == 2:
-        resid = rng.normal(size=(M, N)).astype(np.float32)
-        C = _dev(resid)
-        enc.wf_gemm_bf16(dA, dW, db, 2, C)
-        enc.wf_check()
-        assert np.max(np.abs(to_np(C) - (ref + resid))) < 2e-5 * math.sqrt(K) + 1e-5
-    else:
-        if mode == 1:
-            ref = O.gelu(ref)
-        C = enc.wf_gemm_bf16(dA, dW, db, mode)
-        enc.wf_check()
-        got = to_np(C)
-        assert np.max(np.abs(got - ref) / (np.abs(ref) + 1.0)) < 2.0 ** -8     # bf16 output rounding
+    if mode == 1:
+        ref = O.gelu(ref)
+    C = enc.wf_gemm_bf16(dA, dW, db, mode)
+    enc.wf_check()
+    got = to_np(C)
+    assert np.max(np.abs(got - ref) / (np.abs(ref) + 1.0)) < 2.0 ** -8     # bf16 output rounding
+    enc.close()
+
+
+def _split_planes(x):
+    """x float32 -> (hi, lo) bf16 CUDA tensors with hi = bf16(x), lo = bf16(x - hi), and hi + lo in float64."""
+    xt = _dev(x)
+    hi = xt.to(torch.bfloat16)
+    lo = (xt - hi.float()).to(torch.bfloat16)
+    return hi, lo, hi.double().cpu().numpy() + lo.double().cpu().numpy()
+
+
+def _row_stats(x64):
+    """[K / 128, M, 2] float32 partial (sum, sum of squares) of every 128 columns."""
+    M, K = x64.shape
+    parts = x64.reshape(M, K // 128, 128)
+    return _dev(np.stack([parts.sum(-1).T, (parts ** 2).sum(-1).T], axis=-1).astype(np.float32))
+
+
+@pytest.mark.parametrize("M,N,K", [(300, 384, 240), (1000, 1536, 512), (129, 256, 64), (4097, 1280, 1280),
+                                   (77, 128, 8), (60, 1280, 5120)])
+def test_tcgen05_residual_gemm_on_split_stream(M, N, K):
+    """x <- x + A W^T + bias with x held as two bf16 planes (16 significant bits), and the row
+    statistics the epilogue leaves for the LayerNorm that follows."""
+    shape = _small("bf16", n_layer=0)
+    enc = make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000)
+    rng = np.random.default_rng(M + N + K)
+    A = I.round_to_bf16(rng.normal(size=(M, K)).astype(np.float32))
+    Wm = I.round_to_bf16((rng.normal(size=(N, K)) / math.sqrt(K)).astype(np.float32))
+    bias = rng.normal(size=N).astype(np.float32)
+    hi, lo, x0 = _split_planes((3.0 * rng.normal(size=(M, N)) + 0.5).astype(np.float32))
+    ref = x0 + A.astype(np.float64) @ Wm.astype(np.float64).T + bias
+    stats = enc.wf_gemm_resid_bf16(_dev(A, torch.bfloat16), _dev(Wm, torch.bfloat16), _dev(bias), hi, lo)
+    enc.wf_check()
+    got = hi.double().cpu().numpy() + lo.double().cpu().numpy()
+    assert float(np.max(np.abs(got - ref) - 2.0 ** -16 * np.abs(ref))) <= 2e-5 * math.sqrt(K) + 1e-5
+    hi64, lo64 = hi.double().cpu().numpy(), lo.double().cpu().numpy()
+    assert float(np.max(np.abs(lo64) - 2.0 ** -8 * np.abs(hi64))) <= 0.0       # lo is the rounding remainder of hi
+    st = stats.cpu().numpy().astype(np.float64)
+    parts = got.reshape(M, N // 128, 128)
+    assert np.max(np.abs(st[..., 0] - parts.sum(-1).T)) < 1e-5 * np.abs(parts).sum(-1).max()
+    assert np.max(np.abs(st[..., 1] / (parts ** 2).sum(-1).T - 1.0)) < 1e-5
+    enc.close()
+
+
+@pytest.mark.parametrize("M,N,K", [(300, 384, 256), (1000, 1536, 512), (129, 256, 128), (4097, 3840, 1280), (77, 8, 128)])
+@pytest.mark.parametrize("gelu", [False, True])
+def test_tcgen05_gemm_with_folded_layernorm(M, N, K, gelu):
+    """(gelu of) LN(x) W^T + bias computed as rstd (x_hi W'^T - mean s) + c from the bf16 upper plane
+    of x, the row statistics and the folded weights: tightly against the same formula evaluated in
+    float64 with the library's folded weights, and against the definition on the unrounded x."""
+    shape = _small("bf16", n_layer=0)
+    enc = make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000)
+    rng = np.random.default_rng(M + N + K + 7)
+    # rows of different scale, each with a common mode of the order of its spread (the bf16 rounding of x
+    # is relative to |x|, so a common mode far above the spread would cost accuracy in proportion)
+    x = ((rng.normal(size=(M, K)) + 0.5 * rng.normal(size=(M, 1))) * rng.uniform(0.5, 4.0, size=(M, 1))).astype(np.float32)
+    hi, lo, x64 = _split_planes(x)
+    Wm = I.round_to_bf16((rng.normal(size=(N, K)) / math.sqrt(K)).astype(np.float32))
+    g = (1.0 + 0.2 * rng.normal(size=K)).astype(np.float32)
+    b = (0.2 * rng.normal(size=K)).astype(np.float32)
+    bias = rng.normal(size=N).astype(np.float32)
+    Wg, colsum, cbias = enc.wf_ln_fold(_dev(Wm), _dev(g), _dev(b), _dev(bias))
+    Wg64 = Wg.double().cpu().numpy()
+    assert np.array_equal(Wg.float().cpu().numpy(), I.round_to_bf16((Wm * g[None, :]).astype(np.float32)))
+    assert np.max(np.abs(colsum.cpu().numpy() - Wg64.sum(1))) < 1e-5 * np.abs(Wg64).sum(1).max()
+    assert np.max(np.abs(cbias.cpu().numpy() - (bias + Wm.astype(np.float64) @ b))) < 1e-5
+    out = to_np(enc.wf_gemm_ln_bf16(hi, _row_stats(x64), Wg, colsum, cbias, gelu))
+    enc.wf_check()
+    mu = x64.mean(1, keepdims=True)
+    rstd = 1.0 / np.sqrt(x64.var(1, keepdims=True) + 1e-5)
+    same = rstd * (hi.double().cpu().numpy() @ Wg64.T - mu * Wg64.sum(1)[None, :]) + (bias + Wm.astype(np.float64) @ b)[None, :]
+    ref = O.layer_norm(x64, g, b) @ Wm.astype(np.float64).T + bias
+    if gelu:
+        same, ref = O.gelu(same), O.gelu(ref)
+    assert np.max(np.abs(out - same) / (np.abs(same) + 1.0)) < 2.0 ** -8 + 1e-3      # bf16 output rounding (+ GELU form)
+    assert np.max(np.abs(out - ref) / (np.abs(ref) + 1.0)) < 2.5e-2                   # + bf16 rounding of x and of W gamma
     enc.close()
 
 
@@ -215,55 +284,39 @@ def test_gelu_epilogue_pointwise():
 
 @pytest.mark.parametrize("mode", [0, 2])
 def test_tcgen05_gemm_ragged_last_tile_repeated(mode):
-    """M leaves whole 32-row groups of the last tile outside the matrix and N leaves 32-column
+    """M leaves whole 32-row groups of the last tile outside the matrix and N leaves 64-column
     pieces outside: the epilogue warps that own them store nothing there, and must still not
-    reuse a staging buffer that the previous tile's last copy is reading.  That is a race, so
-    the launch is repeated; every repetition is compared in full (on the device)."""
+    reuse a staging buffer that the previous tile's last copy is reading (mode 0: plain bf16
+    output; mode 2: the residual update on the split stream, which also fetches through those
+    buffers).  That is a race, so the launch is repeated; every repetition is compared in full
+    (on the device)."""
     shape = _small("bf16", n_layer=0)
     enc = make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000)
-    M, N, K = 20000, 1184, 640
+    M, N, K = 20000, (1184 if mode == 0 else 1152), 640
     rng = np.random.default_rng(5)
     A = I.round_to_bf16(rng.normal(size=(M, K)).astype(np.float32))
     Wm = I.round_to_bf16((rng.normal(size=(N, K)) / math.sqrt(K)).astype(np.float32))
     bias = rng.normal(size=N).astype(np.float32)
-    resid = rng.normal(size=(M, N)).astype(np.float32)
-    ref = A.astype(np.float64) @ Wm.astype(np.float64).T + bias + (resid if mode == 2 else 0.0)
-    d_ref, d_resid = _dev(ref.astype(np.float32)), _dev(resid)
+    hi0, lo0, x0 = _split_planes(rng.normal(size=(M, N)).astype(np.float32))
+    ref = A.astype(np.float64) @ Wm.astype(np.float64).T + bias + (x0 if mode == 2 else 0.0)
+    d_ref = _dev(ref.astype(np.float32))
     dA, dW, db = _dev(A, torch.bfloat16), _dev(Wm, torch.bfloat16), _dev(bias)
-    worst = 0.0
+    worst, first = 0.0, None
     for _ in range(25):
         if mode == 2:
-            C = d_resid.clone()
-            enc.wf_gemm_bf16(dA, dW, db, 2, C)
+            hi, lo = hi0.clone(), lo0.clone()
+            stats = enc.wf_gemm_resid_bf16(dA, dW, db, hi, lo)
+            err = (hi.float() + lo.float() - d_ref).abs()
+            if first is None:
+                first = (hi, lo, stats)
+            else:   # no atomics anywhere: every repetition reproduces every bit
+                assert torch.equal(hi, first[0]) and torch.equal(lo, first[1]) and torch.equal(stats, first[2])
         else:
-            C = enc.wf_gemm_bf16(dA, dW, db, 0)
-        err = (C.float() - d_ref).abs()
+            err = (enc.wf_gemm_bf16(dA, dW, db, 0).float() - d_ref).abs()
         worst = max(worst, float((err / (d_ref.abs() + 1.0)).max()) if mode == 0 else float(err.max()))
     enc.wf_check()
-    assert worst < (2.0 ** -8 if mode == 0 else 2e-5 * math.sqrt(K) + 1e-5), worst
+    assert worst < (2.0 ** -8 if mode == 0 else 2e-5 * math.sqrt(K) + 1e-5 + 2.0 ** -14), worst
     enc.close()
-
-
-@pytest.mark.parametrize("M,N,K", [(4097, 1280, 1280), (300, 256, 5120), (20000, 1280, 640)])
-def test_tcgen05_gemm_tail_split_matches_fp64(M, N, K, monkeypatch):
-    """Residual GEMM with the K split of the last partial round of tiles switched on (85 tiles on
-    74 CTA pairs; fewer tiles than pairs; a split limited by the number of K blocks)."""
-    monkeypatch.setenv("WF_GEMM_TAIL_SPLIT", "1")
-    shape = _small("bf16", n_layer=0)
-    enc = make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000)
-    rng = np.random.default_rng(M + N + K)
-    A = I.round_to_bf16(rng.normal(size=(M, K)).astype(np.float32))
-    Wm = I.round_to_bf16((rng.normal(size=(N, K)) / math.sqrt(K)).astype(np.float32))
-    bias = rng.normal(size=N).astype(np.float32)
-    resid = rng.normal(size=(M, N)).astype(np.float32)
-    ref = A.astype(np.float64) @ Wm.astype(np.float64).T + bias + resid
-    C = _dev(resid)
-    enc.wf_gemm_bf16(_dev(A, torch.bfloat16), _dev(Wm, torch.bfloat16), _dev(bias), 2, C)
-    enc.wf_check()
-    assert np.max(np.abs(to_np(C) - ref)) < 2e-5 * math.sqrt(K) + 1e-5
-    enc.close()
-    monkeypatch.delenv("WF_GEMM_TAIL_SPLIT")
-    make_encoder(shape, I.encoder_weights(0, shape), 1, 64, 1000).close()     # back to the default
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])

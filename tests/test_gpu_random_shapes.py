@@ -26,24 +26,47 @@ def enc():
 
 
 def test_gemm_random_shapes(enc):
+    """mode 0 / 1: plain and GELU epilogue; 2: residual update on the split stream (N a multiple of
+    128); 3: LayerNorm folded into the GEMM (K a multiple of 128)."""
     rng = np.random.default_rng(100)
-    for _ in range(120):
+    for _ in range(160):
         M = max(1, int(rng.choice([1, 7, 31, 127, 128, 129, 255, 257, 300, 1000, 4097, 9000, 20000])) + int(rng.integers(-3, 4)))
-        N, K, mode = 8 * int(rng.integers(1, 200)), 8 * int(rng.integers(1, 200)), int(rng.integers(0, 3))
+        N, K, mode = 8 * int(rng.integers(1, 200)), 8 * int(rng.integers(1, 200)), int(rng.integers(0, 4))
+        if mode == 2:
+            N = 128 * int(rng.integers(1, 13))
+        if mode == 3:
+            K = 128 * int(rng.integers(1, 11))
         A = torch.randn(M, K, device="cuda").to(torch.bfloat16)
         W = (torch.randn(N, K, device="cuda") / math.sqrt(K)).to(torch.bfloat16)
         b = torch.randn(N, device="cuda")
         ref = A.float() @ W.float().T + b
         outs = []
+        if mode == 3:
+            stats = torch.stack([A.float().view(M, K // 128, 128).sum(-1).T, (A.float() ** 2).view(M, K // 128, 128).sum(-1).T],
+                                dim=-1).contiguous()
+            ones, zeros = torch.ones(K, device="cuda"), torch.zeros(K, device="cuda")
+            Wg, colsum, cbias = enc.wf_ln_fold(W.float(), ones, zeros, b)
+            assert torch.equal(Wg, W)
+            mu = A.float().mean(1, keepdim=True)
+            ref = (A.float() - mu) / torch.sqrt(A.float().var(1, unbiased=False, keepdim=True) + 1e-5) @ W.float().T + b
         for _ in range(3):
             if mode == 2:
-                C = torch.ones(M, N, device="cuda")
-                enc.wf_gemm_bf16(A, W, b, 2, C)
-                outs.append(C)
+                hi, lo = torch.ones(M, N, device="cuda").to(torch.bfloat16), torch.full((M, N), 2.0 ** -10, device="cuda").to(torch.bfloat16)
+                st = enc.wf_gemm_resid_bf16(A, W, b, hi, lo)
+                outs.append(torch.cat([hi.float() + lo.float(), st[..., 0].T, st[..., 1].T], dim=1))
+            elif mode == 3:
+                outs.append(enc.wf_gemm_ln_bf16(A, stats, Wg, colsum, cbias, False))
             else:
                 outs.append(enc.wf_gemm_bf16(A, W, b, mode))
-        ref = ref + 1.0 if mode == 2 else torch.nn.functional.gelu(ref) if mode == 1 else ref
-        err = float(((outs[0].float() - ref).abs() / (ref.abs() + 1.0)).max())
+        got = outs[0]
+        if mode == 2:
+            ref = ref + 1.0 + 2.0 ** -10
+            sums = got[:, N:N + N // 128].sum(1)
+            assert float(((sums - got[:, :N].sum(1)).abs() / (got[:, :N].abs().sum(1) + 1.0)).max()) < 1e-5, (M, N, K)
+            got = got[:, :N]
+        elif mode == 1:
+            ref = torch.nn.functional.gelu(ref)
+        err = float(((got.float() - ref).abs() / (ref.abs() + 1.0)).max())
         assert all(torch.equal(outs[0], o) for o in outs[1:]), (M, N, K, mode)
         assert err < (2e-4 * math.sqrt(K) if mode == 2 else 2.0 ** -7), (M, N, K, mode, err)
     enc.wf_check()
