@@ -147,6 +147,14 @@ wf_status wf_encode_host(wf_encoder *enc, const float *audio_host, const long *l
  * up since the last check, WF_ERR_CUDA if the stream is in error, else WF_OK. */
 wf_status wf_check(wf_encoder *enc, void *stream);
 
+/* Exercises the failure path behind WF_ERR_DEVICE_TIMEOUT without any fault: enqueues a one-warp
+ * kernel that waits, through the same bounded wait as the GEMM and attention kernels but with
+ * `poll_limit` polls (1 .. 2^20), on a barrier that is never signalled.  The wait runs out, the
+ * kernel records it and ends normally; the next wf_check on this handle returns
+ * WF_ERR_DEVICE_TIMEOUT (and clears the record), and the handle stays fully usable.
+ * (Every wait of the paper's encoding stage as built here, Sec. 3.2 "Operations", is of this kind.) */
+wf_status wf_selftest_wait_timeout(wf_encoder *enc, unsigned poll_limit, void *stream);
+
 wf_status wf_encoder_destroy(wf_encoder *enc);
 const char *wf_last_error(const wf_encoder *enc);
 
@@ -293,9 +301,12 @@ wf_status wf_beam_pruner_destroy(wf_beam_pruner *p);
  * Limits: B <= 256 and M <= 65,536, else WF_ERR_CAPACITY.  No cudaMalloc, cudaFree or other
  * allocating call is made.  The first call on a device looks up the array's device address
  * (once per device, with that device current); make that first call outside any stream
- * capture.  All calls on a device share the array and each overwrites what it reads, so
- * calls are safe back to back on one stream, but calls that may overlap on the GPU (different
- * streams without ordering between them) race on it. */
+ * capture.  A call on a stream that is being captured is rejected (WF_ERR_INVALID_ARG): the
+ * index arrays are copied from the call's own stack frame.  That copy makes the host wait for
+ * earlier work on the stream, so unlike the other entry points this one does not return early.
+ * All calls on a device share the array and each overwrites what it reads, so calls are safe
+ * back to back on one stream, but calls that may overlap on the GPU (different streams without
+ * ordering between them) race on it.  Not thread-safe: call it from one host thread at a time. */
 wf_status wf_attention_f32_static(const float *qkv, const int *cu_seqlens, int B, int d_model,
                                   float *out, void *stream);
 

@@ -54,7 +54,7 @@ _PER_LAYER = ("ln1_g", "ln1_b", "wq", "bq", "wk", "wv", "bv", "wo", "bo", "ln2_g
 
 EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_raw_hush", "wf_encode_mel", "wf_encode_host", "wf_check",
            "wf_encoder_destroy", "wf_last_error", "wf_profile_enable", "wf_profile_read",
-           "wf_gemm_bf16", "wf_attention", "wf_cross_kv", "wf_dtw",
+           "wf_gemm_bf16", "wf_gemm_resid_bf16", "wf_ln_fold", "wf_gemm_ln_bf16", "wf_selftest_wait_timeout", "wf_attention", "wf_cross_kv", "wf_dtw",
            "wf_streams_create", "wf_streams_destroy", "wf_streams_length", "wf_streams_push", "wf_encode_streams", "wf_attention_f32_static",
            "wf_beam_pruner_create", "wf_beam_pruner_step", "wf_beam_pruner_state", "wf_beam_pruner_destroy")
 
@@ -80,6 +80,7 @@ def load_library() -> C.CDLL:
     lib.wf_encoder_destroy.argtypes = [vp]
     lib.wf_last_error.argtypes = [vp]
     lib.wf_last_error.restype = C.c_char_p
+    lib.wf_selftest_wait_timeout.argtypes = [vp, C.c_uint, vp]
     lib.wf_profile_enable.argtypes = [vp, C.c_int]
     lib.wf_profile_read.argtypes = [vp, lp, C.POINTER(C.c_double)]
     lib.wf_gemm_bf16.argtypes = [vp, vp, vp, vp, vp, C.c_long, C.c_int, C.c_int, C.c_int, vp]
@@ -254,6 +255,9 @@ class Encoder:
 
     def wf_check(self, stream=None):
         self._check(self.lib.wf_check(self.handle, _stream_ptr(stream)))
+
+    def wf_selftest_wait_timeout(self, poll_limit: int = 4096, stream=None):
+        self._check(self.lib.wf_selftest_wait_timeout(self.handle, poll_limit, _stream_ptr(stream)))
 
     def wf_profile_enable(self, on: bool):
         self._check(self.lib.wf_profile_enable(self.handle, 1 if on else 0))

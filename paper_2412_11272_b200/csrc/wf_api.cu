@@ -805,8 +805,16 @@ wf_status wf_check(wf_encoder* e, void* stream) {
   WF_CUDA(e, cudaMemcpy(&flag, e->err_flag, sizeof(int), cudaMemcpyDeviceToHost));
   if (flag != 0) {
     cudaMemset(e->err_flag, 0, sizeof(int));
-    return fail(e, WF_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel gave up (role code %d: 1-3 GEMM, 11-13 attention)", flag);
+    return fail(e, WF_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel gave up (role code %d: 1-6 GEMM, 11-13 attention, 21 self-test)", flag);
   }
+  return WF_OK;
+}
+
+wf_status wf_selftest_wait_timeout(wf_encoder* e, unsigned poll_limit, void* stream) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  if (poll_limit < 1 || poll_limit > (1u << 20)) return fail(e, WF_ERR_INVALID_ARG, "poll_limit must be in [1, 2^20]");
+  launch_wait_selftest(e->err_flag, poll_limit, (cudaStream_t)stream);
+  WF_CUDA(e, cudaGetLastError());
   return WF_OK;
 }
 

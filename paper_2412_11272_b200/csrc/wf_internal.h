@@ -148,6 +148,7 @@ void launch_gemm_f32(const float* A, long lda, const float* W, long ldw, long M,
 void launch_layernorm(const float* x, const float* g, const float* b, float* out, long M, int d, cudaStream_t s);
 void launch_attention_f32(const float* qkv, float* out, const int* meta, MetaLayout ml, int n_work,
                           int d_model, cudaStream_t s);
+void launch_wait_selftest(int* err_flag, unsigned poll_limit, cudaStream_t s);
 void launch_convert(const float* src, void* dst, long n, int dst_bf16, cudaStream_t s);
 void launch_conv_weight(const float* src /*[out, in, 3]*/, void* dst /*[out, 3*in_ld], zeroed*/, int c_out,
                         int c_in, int in_ld, int dst_bf16, cudaStream_t s);

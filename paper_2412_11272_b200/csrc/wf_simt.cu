@@ -294,6 +294,27 @@ void launch_attention_f32(const float* qkv, float* out, const int* meta, MetaLay
 }
 
 // ---------------------------------------------------------------------------------------------
+// Self-test of the bounded wait every tensor-core kernel of the library relies on: one warp waits,
+// with the same wait routine but a caller-chosen poll limit, on an mbarrier that nobody ever
+// arrives on.  The wait must run out, raise the shared abort flag and return; the kernel then
+// records role code 21 in the device error word and ends normally.  No TMA, no tensor memory.
+__global__ void __launch_bounds__(32) wait_selftest_kernel(int* err_flag, uint32_t poll_limit) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncwarp();
+  const bool ok = ptx::mbar_wait_limited(ptx::smem_u32(&bar), 0, &abort_flag, poll_limit);
+  if (!__all_sync(0xffffffffu, ok) && threadIdx.x == 0) atomicExch(err_flag, 21);
+}
+void launch_wait_selftest(int* err_flag, unsigned poll_limit, cudaStream_t s) {
+  wait_selftest_kernel<<<1, 32, 0, s>>>(err_flag, poll_limit);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Weight conversion at create time.
 template <typename OutT>
 __global__ void convert_kernel(const float* __restrict__ src, OutT* __restrict__ dst, long n) {

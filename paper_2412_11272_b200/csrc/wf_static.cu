@@ -21,6 +21,8 @@ constexpr int kStaticInts = (kStaticMaxBatch + 1) + 2 * kStaticMaxWork;   // 8,9
 // overwrites the part it reads (prefix sums, then work list) before its kernel runs.
 static __device__ __align__(256) int g_static_meta[kStaticInts];
 
+// Device address of the array on each device, looked up on first use.  Plain host state: calls
+// from several host threads at once are not supported.
 constexpr int kMaxDevices = 64;
 int* g_static_meta_ptr[kMaxDevices] = {nullptr};
 
@@ -36,6 +38,12 @@ extern "C" wf_status wf_attention_f32_static(const float* qkv, const int* cu_seq
   for (int i = 0; i < B; ++i)
     if (cu_seqlens[i + 1] <= cu_seqlens[i]) return WF_ERR_INVALID_ARG;
   if (cu_seqlens[B] > kStaticMaxTokens) return WF_ERR_CAPACITY;
+
+  cudaStream_t s = (cudaStream_t)stream;
+  // The index arrays are uploaded from this call's stack frame: a captured copy would outlive it.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) return WF_ERR_CUDA;
+  if (cap != cudaStreamCaptureStatusNone) return WF_ERR_INVALID_ARG;
 
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return WF_ERR_CUDA;
@@ -60,10 +68,11 @@ extern "C" wf_status wf_attention_f32_static(const float* qkv, const int* cu_seq
       ++nw;
     }
   ml.total = ml.attn_work + 2 * nw;
-  cudaStream_t s = (cudaStream_t)stream;
-  // Pageable source: the runtime has taken its copy of host_meta when this call returns.
+  // Pageable source: the runtime has taken its copy of host_meta when this call returns (which
+  // makes the host wait for earlier work on the stream).
   if (cudaMemcpyAsync(meta_dev, host_meta, (size_t)ml.total * sizeof(int), cudaMemcpyHostToDevice, s) != cudaSuccess)
     return WF_ERR_CUDA;
+  cudaGetLastError();  // an error left behind by earlier work is not this launch's
   wf::launch_attention_f32(qkv, out, meta_dev, ml, nw, d_model, s);
   return cudaGetLastError() == cudaSuccess ? WF_OK : WF_ERR_CUDA;
 }

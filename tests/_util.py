@@ -34,6 +34,14 @@ def peak_rel_err(got, ref):
     return float(np.max(np.abs(got - ref)) / np.max(np.abs(ref)))
 
 
+def elementwise_excess(got, ref, rel=3e-2):
+    """max over elements of |got - ref| / (rel |ref| + rel rms(ref row)): at most 1 when every element is
+    within `rel` of its own magnitude plus `rel` of its token's root mean square (covers the channels
+    far below the sequence's peak, which the peak-normalised measure cannot see)."""
+    rms = np.sqrt((ref ** 2).mean(axis=1, keepdims=True))
+    return float((np.abs(got - ref) / (rel * np.abs(ref) + rel * rms)).max())
+
+
 def min_token_cosine(got, ref):
     num = (got * ref).sum(axis=1)
     den = np.linalg.norm(got, axis=1) * np.linalg.norm(ref, axis=1)

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 
 from paper_2412_11272_b200 import inputs as I
-from tests._util import make_encoder, min_token_cosine, oracle_hidden, peak_rel_err, to_np
+from tests._util import elementwise_excess, make_encoder, min_token_cosine, oracle_hidden, peak_rel_err, to_np
 
 pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
@@ -46,6 +46,7 @@ def _run(name, batch, hush_frames, picks, n_ctx=None):
         g = got[cu[i]:cu[i + 1]]
         assert peak_rel_err(g, ref) <= 3e-2, (name, i)
         assert min_token_cosine(g, ref) >= 0.999, (name, i)
+        assert elementwise_excess(g, ref) <= 1.0, (name, i)
     enc.close()
     return got, cu
 

@@ -8,7 +8,7 @@ import pytest
 
 from oracle import wf_oracle as O
 from paper_2412_11272_b200 import inputs as I
-from tests._util import make_encoder, min_token_cosine, oracle_hidden, peak_rel_err, to_np
+from tests._util import elementwise_excess, make_encoder, min_token_cosine, oracle_hidden, peak_rel_err, to_np
 
 pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
@@ -415,8 +415,11 @@ def test_varlen_attention_matches_oracle(dtype):
 # ------------------------------------------------------------------------------ bf16 path
 
 def _check_bf16(got, ref):
+    """The stated bf16 tolerance read as max|err| / max|ref| per sequence and per-token cosine, plus
+    an element-wise bound that also covers channels far below the sequence's peak."""
     assert peak_rel_err(got, ref) <= BF16_REL
     assert min_token_cosine(got, ref) >= BF16_COS
+    assert elementwise_excess(got, ref, BF16_REL) <= 1.0
 
 
 def test_bf16_small_ragged_matches_oracle():
@@ -595,6 +598,33 @@ def test_stream_windows_match_encoding_from_scratch(dtype):
 
 
 # ------------------------------------------------------------------------------ errors and edges
+
+def test_bounded_wait_runs_out_and_is_reported():
+    """The failure path of every bounded device-side wait, exercised without a fault: a one-warp
+    kernel waits with the library's wait routine on a barrier nobody signals; the wait gives up
+    after the requested number of polls, the kernel ends normally, wf_check reports
+    WF_ERR_DEVICE_TIMEOUT once, and the handle then encodes as before."""
+    from paper_2412_11272_b200.binding import WfError
+    shape = _small("bf16", d_model=256, n_head=4, d_mlp=512, n_layer=2)
+    W = I.encoder_weights(11, shape)
+    batch = I.batch_from_lengths(11, [160 * 40, 160 * 121])
+    hush = I.round_to_bf16(I.hush_mel(11, shape.n_mel))
+    enc = make_encoder(shape, W, 2, 200, int(batch.lengths.sum()))
+    before, cu = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush))
+    enc.wf_check()
+    enc.wf_selftest_wait_timeout(2000)
+    with pytest.raises(WfError) as ei:
+        enc.wf_check()
+    assert ei.value.status == "WF_ERR_DEVICE_TIMEOUT"
+    enc.wf_check()                                   # the record was cleared by the failing check
+    after, _ = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush))
+    enc.wf_check()
+    assert torch.equal(before, after)
+    refs = oracle_hidden(batch, shape, W, hush)
+    for i, ref in refs.items():
+        _check_bf16(to_np(after)[cu[i]:cu[i + 1]], ref)
+    enc.close()
+
 
 def test_errors_and_edge_cases():
     from paper_2412_11272_b200.binding import WfError
