@@ -33,10 +33,12 @@ UNIT = "audio-s/s"
 WORKLOAD = "large-v3-shaped bf16 encoder, 64 streams x windows of 1..15 s + 50 hush frames (15 ragged calls per step)"
 N_STREAMS = 64
 ROUNDS = list(range(1, 16))
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from an ncu capture
-# of the current kernels; None until the counters have been re-taken after a kernel change
-TRAFFIC_PER_LAUNCH = None
-TRAFFIC_NOTE = "the block GEMM kernels changed since the last counter capture"
+# dram__bytes_read.sum + dram__bytes_write.sum of the four block GEMMs (QKV, out-projection, FC1, FC2)
+# from one ncu capture of the current kernels at M = 16384; the traffic grows in proportion to M
+# (activations dominate, weights are read once per launch), so it is scaled per token to the mean
+# launch of the benchmark.  Set to None whenever a GEMM kernel changes, until re-captured.
+GEMM_DRAM_BYTES_M16384 = (127.4e6, 160.4e6, 173.5e6, 367.6e6)
+TRAFFIC_NOTE = "DRAM bytes per launch (mean over the four GEMM shapes), scaled per token from the M = 16384 ncu capture"
 SAMPLE_SECONDS = 15         # the CPU oracle is timed on stream 0's full 15 s window (775 tokens)
 
 
@@ -404,7 +406,8 @@ def run_ours(args, rank, world, local_rank):
                      "frac_of_burst": (gemm_tflops / peaks["bf16_burst"]) if gemm_tflops else None,
                      "launches": gemm["launches"],
                      "timing": "CUDA events around every launch of the class, in the profiled pass over the same steps",
-                     "traffic": TRAFFIC_PER_LAUNCH,
+                     "traffic": (sum(GEMM_DRAM_BYTES_M16384) / 16384.0 * args.steps * step_tokens * shape.n_layer / max(gemm["launches"], 1)
+                                 if GEMM_DRAM_BYTES_M16384 else None),
                      "traffic_note": TRAFFIC_NOTE},
     }
     if world == 1:
