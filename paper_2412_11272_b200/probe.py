@@ -1,6 +1,8 @@
-"""Runs one component of the library alone, for timing and for profiler captures.
+"""Runs one component of the library alone, for timing and for profiler captures: the commands
+quoted in the profiler summaries that ship with the library are invocations of this module.
 
-    python -m paper_2412_11272_b200.probe gemm --M 16384 --N 3840 --K 1280 --mode 0
+    python -m paper_2412_11272_b200.probe gemm --M 16384 --N 3840 --K 1280 --mode 0    (modes: 0 bias, 1 + GELU,
+                                         2 residual update on the split stream, 3 / 4 LayerNorm folded in)
     python -m paper_2412_11272_b200.probe attention --n 775 --batch 64
     python -m paper_2412_11272_b200.probe encode --shape large --seconds 3 --batch 16
     python -m paper_2412_11272_b200.probe logmel --seconds 15 --batch 64

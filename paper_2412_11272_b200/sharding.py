@@ -35,6 +35,30 @@ def lpt_partition(costs, world: int) -> list[list[int]]:
     return [sorted(p) for p in parts]
 
 
+def rank_cu_seqlens(tokens, part) -> np.ndarray:
+    """Token prefix sums of the sub-batch a rank encodes: its sequences `part` (indices into the
+    whole batch, ascending) keep their relative order."""
+    t = np.asarray(tokens, dtype=np.int64)[list(part)]
+    return np.concatenate([[0], np.cumsum(t)]).astype(np.int64)
+
+
+def reassemble_packed(shards, parts, tokens) -> np.ndarray:
+    """Packed hidden states of the whole batch, rows in the original sequence order, from every
+    rank's packed output (`shards[r]` is rank r's [sum of its tokens, d] array, `parts[r]` its
+    sequence indices).  This is the optional gather behind a strong-scaling split: the sequences
+    themselves never exchange anything."""
+    tokens = np.asarray(tokens, dtype=np.int64)
+    cu = np.concatenate([[0], np.cumsum(tokens)])
+    d = shards[0].shape[1]
+    out = np.empty((int(cu[-1]), d), dtype=shards[0].dtype)
+    for shard, part in zip(shards, parts):
+        local = rank_cu_seqlens(tokens, part)
+        assert shard.shape[0] == local[-1], "a rank's output does not match its sequences"
+        for j, i in enumerate(part):
+            out[cu[i]:cu[i + 1]] = shard[local[j]:local[j + 1]]
+    return out
+
+
 def max_over_ranks(value: float, device="cpu") -> float:
     """The slowest rank's time: what a multi-GPU throughput has to be computed from."""
     if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:

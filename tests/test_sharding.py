@@ -1,5 +1,6 @@
 """Multi-rank host logic on CPU (gloo, world size 2): stream ownership, the max-over-ranks
-timing reduction, and the cost-balanced partition of one ragged batch."""
+timing reduction, and the cost-balanced partition of one ragged batch with the per-rank
+cu_seqlens and the reassembly of the packed rows."""
 import os
 
 import numpy as np
@@ -27,9 +28,22 @@ def _worker(rank, world, port, out_dir):
         all_parts = [None] * world
         dist.all_gather_object(all_parts, mine)
         loads = [float(cost[p].sum()) for p in all_parts]
+        # strong scaling of ONE ragged batch: every rank "encodes" its sequences (a stand-in that
+        # marks each row with its sequence and position), the packed outputs are gathered and put
+        # back into the order a single-rank call would have produced
+        tokens = I.tokens_of(lengths)
+        cu_mine = sharding.rank_cu_seqlens(tokens, mine)
+        rows = np.concatenate([np.stack([np.full(tokens[i], i), np.arange(tokens[i])], axis=1) for i in mine])
+        assert rows.shape[0] == cu_mine[-1] and list(np.diff(cu_mine)) == [int(tokens[i]) for i in mine]
+        shards = [None] * world
+        dist.all_gather_object(shards, rows)
+        whole = sharding.reassemble_packed(shards, all_parts, tokens)
+        expect = np.concatenate([np.stack([np.full(t, i), np.arange(t)], axis=1) for i, t in enumerate(tokens)])
+        reassembled = float(np.array_equal(whole, expect))
         np.save(os.path.join(out_dir, f"r{rank}.npy"),
                 np.array([slowest, float(sorted(sum(gathered, [])) == list(range(4 * world))),
-                          float(sorted(sum(all_parts, [])) == list(range(64))), max(loads) / (sum(loads) / world)]))
+                          float(sorted(sum(all_parts, [])) == list(range(64))), max(loads) / (sum(loads) / world),
+                          reassembled]))
     finally:
         dist.destroy_process_group()
 
@@ -39,7 +53,8 @@ def test_two_ranks_on_gloo(tmp_path):
     port = 29500 + (os.getpid() % 2000)
     mp.spawn(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
     for rank in range(world):
-        slowest, disjoint, covered, imbalance = np.load(tmp_path / f"r{rank}.npy")
+        slowest, disjoint, covered, imbalance, reassembled = np.load(tmp_path / f"r{rank}.npy")
+        assert reassembled == 1.0              # per-rank cu_seqlens and the gather restore the single-rank row order
         assert slowest == 15.0                 # the max, on every rank
         assert disjoint == 1.0 and covered == 1.0
         assert imbalance < 1.05                # LPT balances 64 ragged sequences within 5 %
