@@ -67,3 +67,20 @@ def test_synthetic_attention_costs_recover_a_monotone_alignment():
     assert np.all(np.diff(start) >= 0) and start[0] == 0
     centres = np.argmin(C - 0 * C, axis=1)
     assert np.mean(np.abs(start - centres)) < 30            # starts sit near (before) the band centres
+
+
+def test_tie_order_on_hand_worked_matrices():
+    """The stated tie order (diagonal, then the step in the token index, then the step in the frame
+    index), on matrices small enough to fill in by hand.
+    All ones, 2 x 3: D = [[1, 2, 3], [2, 2, 3]].  The last cell sees diagonal D[0,1] = 2 and left
+    D[1,1] = 2 (up is 3): the tie goes to the diagonal, so the path is (0,0) (0,1) (1,2) and token 1
+    starts at frame 2 (a left-first rule would give (0,0) (1,1) (1,2) and frame 1)."""
+    total, path, start = D.dtw(np.ones((2, 3), np.float32))
+    assert total == 3.0 and path == [(0, 0), (0, 1), (1, 2)] and list(start) == [0, 2]
+    # C = [[5, -1], [-1, 0]]: D = [[5, 4], [4, 4]]; the last cell sees diagonal 5, up 4, left 4: the tie
+    # between the two steps goes to the step in the token index, i.e. the predecessor (0, 1)
+    total, path, start = D.dtw(np.array([[5, -1], [-1, 0]], np.float32))
+    assert total == 4.0 and path == [(0, 0), (0, 1), (1, 1)] and list(start) == [0, 1]
+    # all zeros, 3 x 3: everything ties, the diagonal wins at every cell
+    total, path, start = D.dtw(np.zeros((3, 3), np.float32))
+    assert total == 0.0 and path == [(0, 0), (1, 1), (2, 2)] and list(start) == [0, 1, 2]

@@ -517,6 +517,20 @@ def test_dtw_matches_oracle_bit_for_bit():
             assert total[b] == t_ref                               # same float32 additions, same order
             assert np.array_equal(start[off:off + len(s_ref)], s_ref), (batch, b)
             off += len(s_ref)
+    # ties: matrices whose cells tie by construction (constant, small integers), where the stated order
+    # (diagonal, then the token step, then the frame step) decides the path
+    rng = np.random.default_rng(8)
+    ties = [np.ones((2, 3), np.float32), np.array([[5, -1], [-1, 0]], np.float32), np.zeros((3, 3), np.float32),
+            np.zeros((37, 150), np.float32), rng.integers(0, 3, size=(60, 200)).astype(np.float32)]
+    start, total = enc.wf_dtw(_dev(np.concatenate([c.reshape(-1) for c in ties])), [c.shape[0] for c in ties],
+                              [c.shape[1] for c in ties])
+    enc.wf_check()
+    start, total = start.cpu().numpy(), total.cpu().numpy()
+    off = 0
+    for b, c in enumerate(ties):
+        t_ref, _, s_ref = dtw_oracle.dtw(c)
+        assert total[b] == t_ref and np.array_equal(start[off:off + len(s_ref)], s_ref), b
+        off += len(s_ref)
     enc.close()
 
 
