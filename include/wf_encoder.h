@@ -85,13 +85,16 @@ typedef struct {
  * the stated capacities.  Synchronises `stream` before returning.  Fails with
  * WF_ERR_UNSUPPORTED_ARCH on a device that is not compute capability 10.x.
  * (Operation: the encoder of Sec. 1.1 / Sec. 2.3; weights are caller-provided.)
- * Two tuning switches of the WF_BF16 path are read from the environment here and kept in the
+ * Three tuning switches of the WF_BF16 path are read from the environment here and kept in the
  * handle (a later create with another environment does not change this one):
  *   WF_PDL=0               launch kernels plainly instead of with programmatic stream
  *                          serialization (on by default: a kernel's set-up overlaps the tail of
  *                          the kernel before it);
- *   WF_GEMM_SMALL_TILES=0  never use 128 x 128 single-CTA tiles for small GEMMs.
- * Neither changes what is computed.  Results are bit-reproducible from call to call: no kernel of
+ *   WF_GEMM_SMALL_TILES=0  never use 128 x 128 single-CTA tiles for small GEMMs;
+ *   WF_GEMM_SPLIT_K=n      split the K range of a GEMM with few tiles over a cluster of CTAs when K
+ *                          has at least n blocks of 64 (default 64; 0 = never).
+ * None of them changes what is computed beyond float32 rounding order (which is fixed for a
+ * given setting).  Results are bit-reproducible from call to call: no kernel of
  * the encoder combines partial results in an order that varies. */
 wf_status wf_encoder_create(const wf_config *cfg, const wf_weights *w, void *stream,
                             wf_encoder **out);

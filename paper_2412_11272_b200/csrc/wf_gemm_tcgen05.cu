@@ -35,22 +35,21 @@ constexpr int kXLook = 1;
 constexpr int kSmemBudget = 224 * 1024;  // operand stages + epilogue staging
 
 // Shared-memory plan of a CTA that stages 128 x 64 of A and BROWS x 64 of W per stage.
-template <int BROWS, int EPI>
+template <int BROWS, int EPI, int XS = kXSets>
 struct SmemPlan {
   static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = BROWS * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStagingPerWarp = EPI == kEpiResidSplit ? kXSets * 8192 : 2 * 4096;
+  static constexpr int kStagingPerWarp = EPI == kEpiResidSplit ? XS * 8192 : 2 * 4096;
   static constexpr int kStages = (kSmemBudget - 4 * kStagingPerWarp) / kStageBytes;
   static constexpr int kStagingOffset = kStages * kStageBytes;
   static constexpr int kBarOffset = kStagingOffset + 4 * kStagingPerWarp;
-  // barriers: full[kStages], empty[kStages], tfull[2], tempty[2], xld[4][kXSets]; then the tensor
-  // memory slot and the abort flag
+  // barriers: full[kStages], empty[kStages], tfull[2], tempty[2], xld[4][kXSets] (XS <= kXSets of them
+  // used per warp); then the tensor memory slot and the abort flag
   static constexpr int kNumBars = 2 * kStages + 4 + 4 * kXSets;
   static constexpr int kSmemBytes = kBarOffset + 8 * kNumBars + 16 + 1024;  // + alignment slack
   static_assert(kStages >= 3 && 8 * kNumBars + 16 <= 256, "shared-memory plan");
 };
-constexpr int kMaxGemmSmem = kSmemBudget + 256 + 1024;
 
 __host__ __device__ constexpr bool epi_is_ln(int epi) { return epi == kEpiLnBias || epi == kEpiLnBiasGelu; }
 
@@ -70,6 +69,31 @@ __device__ __forceinline__ float2 row_norm(const EpiParams& ep, long row, long M
   const float var = fmaxf(fmaf(s2, inv, -mean * mean), 0.f);
   const float rstd = rsqrtf(var + 1e-5f);
   return make_float2(rstd, -rstd * mean);
+}
+
+// Partial accumulators of a tile whose K range was split over the CTAs of a cluster (the single-CTA
+// kernel's small-M variant): CTAs 1 .. n of the cluster leave their 128 x 128 float32 accumulators
+// in the shared memory of CTA 0 (its operand stages, idle by then), which adds them to its own in
+// rank order before the epilogue arithmetic.  Layout of one partial (64 KB): row r at r * 512
+// bytes, its 16-byte chunk c at position (c & ~7) | ((c & 7) ^ (r & 7)).
+struct Partials {
+  uint32_t base;  // shared-memory address of the first partial (in the CTA that reads them)
+  int n;          // how many (0: none)
+};
+__device__ __forceinline__ uint32_t partial_addr(uint32_t base, int p, int row, int chunk) {
+  return base + (uint32_t)p * 65536u + (uint32_t)row * 512u + (uint32_t)(((chunk & ~7) | ((chunk & 7) ^ (row & 7))) << 4);
+}
+// acc (32 columns starting at tile column c0, accumulator row `row`) += the partials, in rank order
+__device__ __forceinline__ void add_partials(const Partials& ps, int row, int c0, uint32_t (&acc)[32]) {
+  for (int p = 0; p < ps.n; ++p) {
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+      uint32_t q[4];
+      ld_shared_v4(partial_addr(ps.base, p, row, (c0 >> 2) + g), q[0], q[1], q[2], q[3]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[4 * g + i] = __float_as_uint(__uint_as_float(acc[4 * g + i]) + __uint_as_float(q[i]));
+    }
+  }
 }
 
 // Epilogue arithmetic of 32 accumulator columns starting at col0 (col0 + 32 <= padded N is not
@@ -144,7 +168,7 @@ __device__ __forceinline__ void conv2_store32(const EpiParams& ep, int2 d, int c
 template <int BN, int EPI>
 __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtensorMap* tmap_c, uint32_t t_row, int m0,
                                               int n0, long M, int N, int K, int quarter, int lane, uint32_t stage_base,
-                                              uint32_t& piece) {
+                                              uint32_t& piece, const Partials ps = Partials{0u, 0}) {
   const long row = (long)m0 + quarter * 32 + lane;
   if (EPI == kEpiConv2) {
     const int2 d = row < M ? ep.row_dst[row] : make_int2(-1, 0);
@@ -179,6 +203,7 @@ __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtenso
         float v[32];
         tmem_ld_32x32(t_row + c * 64 + hf * 32, a32);
         tmem_ld_wait();
+        if (ps.n > 0) add_partials(ps, quarter * 32 + lane, c * 64 + hf * 32, a32);
         bias_act32<EPI>(ep, n0 + c * 64 + hf * 32, N, a32, v, nrm);
         if (EPI == kEpiConv1 && !valid) {
 #pragma unroll
@@ -224,16 +249,19 @@ __device__ __forceinline__ bool piece_xy(const XWalk& w, uint32_t p, long M, int
   y = (int)(t / w.num_n) * w.tile_rows + w.row_off;
   return x < N && y < M;
 }
-// One lane: fetch the old x_hi / x_lo values of piece p into its staging set.
+// One lane: fetch the old x_hi / x_lo values of piece p into its staging set (XS sets per warp, the
+// fetch running XL pieces ahead of the piece being processed).
+template <int XS = kXSets, int XL = kXLook>
 __device__ __forceinline__ void x_fetch(const XWalk& w, uint32_t p, long M, int N, const CUtensorMap* t_hi,
                                         const CUtensorMap* t_lo, uint32_t stage_base, uint32_t xbar0, uint32_t& armed) {
   int x, y;
   if (!piece_xy(w, p, M, N, x, y)) return;
-  const uint32_t set = p % kXSets;
-  // The set was last used by piece p - kXSets.  This runs while piece p - kXLook is current, after
-  // the groups of all earlier pieces were committed: at most kXSets - kXLook - 1 of them may still
-  // be reading shared memory.
-  bulk_wait_read<kXSets - kXLook - 1>();
+  const uint32_t set = p % XS;
+  // The set was last used by piece p - XS.  This runs while piece p - XL is current, after the
+  // groups of all earlier pieces were committed: at most XS - XL - 1 of them may still be reading
+  // shared memory.
+  static_assert(XS - XL - 1 >= 0, "the fetch may not run further ahead than there are sets");
+  bulk_wait_read<XS - XL - 1>();
   mbar_arrive_expect_tx(xbar0 + 8u * set, 8192);
   tma_load_2d(stage_base + set * 8192u, t_hi, x, y, xbar0 + 8u * set);
   tma_load_2d(stage_base + set * 8192u + 4096u, t_lo, x, y, xbar0 + 8u * set);
@@ -246,20 +274,20 @@ struct XState {
 };
 // One tile: x <- x + acc + bias in place in shared memory, pieces stored back by TMA, the row's
 // (sum, sum of squares) over each 128 columns written to stats_out.  False after a timed-out wait.
-template <int BN>
+template <int BN, int XS = kXSets, int XL = kXLook>
 __device__ __forceinline__ bool epilogue_tile_split(const EpiParams& ep, const CUtensorMap* t_hi, const CUtensorMap* t_lo,
                                                     uint32_t t_row, int m0, int n0, long M, int N, int quarter, int lane,
                                                     uint32_t stage_base, uint32_t xbar0, const XWalk& w, XState& st,
-                                                    volatile int* abort_flag) {
+                                                    volatile int* abort_flag, const Partials ps = Partials{0u, 0}) {
   const long row = (long)m0 + quarter * 32 + lane;
   float s1 = 0.f, s2 = 0.f;
 #pragma unroll 1
   for (int c = 0; c < BN / 64; ++c) {
     const uint32_t p = st.piece;
-    if (lane == 0) x_fetch(w, p + kXLook, M, N, t_hi, t_lo, stage_base, xbar0, st.armed);
+    if (lane == 0) x_fetch<XS, XL>(w, p + XL, M, N, t_hi, t_lo, stage_base, xbar0, st.armed);
     const bool valid = n0 + c * 64 < N && (long)m0 + quarter * 32 < M;
     if (valid) {
-      const uint32_t set = p % kXSets;
+      const uint32_t set = p % XS;
       const uint32_t buf = stage_base + set * 8192u;
       bool ok = mbar_wait(xbar0 + 8u * set, (st.phase >> set) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
@@ -272,6 +300,7 @@ __device__ __forceinline__ bool epilogue_tile_split(const EpiParams& ep, const C
         float v[32];
         tmem_ld_32x32(t_row + c * 64 + hf * 32, a32);
         tmem_ld_wait();
+        if (ps.n > 0) add_partials(ps, quarter * 32 + lane, c * 64 + hf * 32, a32);
         bias_act32<kEpiResidSplit>(ep, n0 + c * 64 + hf * 32, N, a32, v, make_float2(0.f, 0.f));
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -487,6 +516,173 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 2 * BN);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Small-M variant of the single-CTA kernel: one 128 x 128 tile per CLUSTER of `split` CTAs, each
+// CTA accumulating its share of the K range (so that a few tiles still draw their weights through
+// many SMs: one SM takes in about 100 GB/s, and ten tiles of K = 5120 would otherwise stream a
+// 13 MB weight matrix through ten SMs).  The partial accumulators meet in CTA 0's shared memory
+// through distributed shared memory (see Partials) and are added in rank order: the result does
+// not depend on timing.  Two cluster barriers separate the phases; every thread reaches both,
+// also after a timed-out wait.  The hand-over costs several microseconds per launch, so the
+// launcher only splits GEMMs with a long K range (64 K blocks = K >= 4096 by default: FC2).
+template <int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_splitk_kernel(
+    const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+    const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_c2, long M, int N, int K,
+    EpiParams ep, int* err_flag, int split) {
+  constexpr int BN = 128;
+  // one staging set per warp for the residual epilogue (a warp has only two pieces to update): that
+  // leaves six operand stages, 192 KB, for up to three partial accumulators
+  using Cfg = SmemPlan<BN, EPI, 1>;
+  static_assert(Cfg::kStagingOffset >= 3 * 65536, "three partial accumulators fit in the operand stages");
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + Cfg::kBarOffset;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (Cfg::kStages + s); };
+  const uint32_t tfull_bar = bar_base + 8u * (2 * Cfg::kStages);
+  const uint32_t xbar_base = bar_base + 8u * (2 * Cfg::kStages + 4);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + Cfg::kBarOffset + 8 * Cfg::kNumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + Cfg::kBarOffset + 8 * Cfg::kNumBars + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();
+  const int tile = (int)blockIdx.x / split;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(tfull_bar, 1);
+    for (int i = 0; i < 4 * kXSets; ++i) mbar_init(xbar_base + 8u * i, 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), BN);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();  // nothing of another CTA is touched before the first cluster barrier below
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();  // everything above overlapped the previous kernel's tail; its output is needed from here on
+  griddep_launch_dependents();
+
+  const int num_n = (N + BN - 1) / BN;
+  const int num_k = (K + kBK - 1) / kBK;
+  const int m0 = (tile / num_n) * kBM, n0 = (tile % num_n) * BN;
+  const int kb0 = rank * num_k / split, kb1 = (rank + 1) * num_k / split;  // split <= num_k: never empty
+  const int quarter = warp & 3;
+  const uint32_t stage_base = smem_base + Cfg::kStagingOffset + (uint32_t)((warp - 2) * Cfg::kStagingPerWarp);
+  const uint32_t xbar0 = xbar_base + 8u * (uint32_t)((warp - 2) * kXSets);
+  const XWalk walk{tile, 1 << 30, tile + 1, num_n, kBM, quarter * 32, BN, BN / 64};
+  XState xs{0u, 0u, 0u};
+  bool acc_ok = true;  // epilogue warps: this CTA's accumulator is complete
+
+  // ---- phase 1: this CTA's share of the K range
+  if (warp == 0) {
+    if (lane == 0) {
+      prefetch_tmap(&tmap_a);
+      prefetch_tmap(&tmap_b);
+      int stage = 0;
+      uint32_t phase = 0, armed = 0, armed_parity = 0;
+      bool ok = true;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+        mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageBytes);
+        const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
+        tma_load_2d(sa, &tmap_a, kb * kBK, m0, full_bar(stage));
+        tma_load_2d(sa + Cfg::kABytes, &tmap_b, kb * kBK, n0, full_bar(stage));
+        armed |= 1u << stage;
+        armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+        if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) {
+        atomicExch(err_flag, 7);
+        drain_stages(full_bar(0), Cfg::kStages, armed, armed_parity);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN, 0, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
+        const uint64_t adesc = umma_desc_k_sw128(sa);
+        const uint64_t bdesc = umma_desc_k_sw128(sa + Cfg::kABytes);
+#pragma unroll
+        for (int k = 0; k < kBK / 16; ++k) umma_bf16(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > kb0 || k != 0) ? 1u : 0u);
+        umma_commit(empty_bar(stage));
+        if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
+      }
+      if (ok) umma_commit(tfull_bar);
+      else atomicExch(err_flag, 8);
+    }
+  } else {
+    if (EPI == kEpiResidSplit && rank == 0 && lane == 0) {
+      prefetch_tmap(&tmap_c);
+      prefetch_tmap(&tmap_c2);
+    }
+    acc_ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar, 0, abort_flag));
+    if (!acc_ok && lane == 0) atomicExch(err_flag, 9);
+    tc_fence_after();
+  }
+  // every CTA's accumulator is complete and its operand stages are idle (all its MMAs have completed)
+  tc_fence_before();
+  cluster_sync_all();
+
+  // ---- phase 2: CTAs 1 .. split - 1 hand their accumulators to CTA 0
+  if (warp >= 2 && rank > 0) {
+    tc_fence_after();
+    const int row = quarter * 32 + lane;
+    const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+      uint32_t a32[32];
+      tmem_ld_32x32(t_row + c * 32, a32);
+      tmem_ld_wait();
+#pragma unroll
+      for (int g = 0; g < 8; ++g)
+        st_cluster_v4(map_to_cta(partial_addr(smem_base, rank - 1, row, 8 * c + g), 0), a32[4 * g], a32[4 * g + 1],
+                      a32[4 * g + 2], a32[4 * g + 3]);
+    }
+  }
+  cluster_sync_all();  // release / acquire: the partials are visible in CTA 0
+
+  // ---- phase 3: CTA 0 adds them up and runs the epilogue
+  if (warp >= 2 && rank == 0) {
+    tc_fence_after();
+    const Partials ps{smem_base, split - 1};
+    const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    uint32_t piece = 0;
+    bool ok = true;
+    if constexpr (EPI == kEpiResidSplit)
+      ok = epilogue_tile_split<BN, 1, 0>(ep, &tmap_c, &tmap_c2, t_row, m0, n0, M, N, quarter, lane, stage_base, xbar0, walk, xs,
+                                         abort_flag, ps);
+    else
+      epilogue_tile<BN, EPI>(ep, &tmap_c, t_row, m0, n0, M, N, K, quarter, lane, stage_base, piece, ps);
+    if (!ok && lane == 0) {
+      atomicExch(err_flag, 9);
+      x_drain(xbar0, xs);
+    }
+    if (lane == 0) bulk_wait_all();  // every store this lane issued has completed
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, BN);
   }
 }
 
@@ -711,6 +907,12 @@ static cudaError_t configure_one() {
 }
 
 template <int EPI>
+static cudaError_t configure_splitk() {
+  return cudaFuncSetAttribute(gemm_bf16_splitk_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              SmemPlan<128, EPI, 1>::kSmemBytes);
+}
+
+template <int EPI>
 static cudaError_t configure_pair() {
   cudaError_t e = cudaFuncSetAttribute(gemm_bf16_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        SmemPlan<128, EPI>::kSmemBytes);
@@ -733,6 +935,11 @@ cudaError_t gemm_bf16_configure() {
   if ((e = configure_one<kEpiLnBias>()) != cudaSuccess) return e;
   if ((e = configure_one<kEpiLnBiasGelu>()) != cudaSuccess) return e;
   if ((e = configure_one<kEpiResidSplit>()) != cudaSuccess) return e;
+  if ((e = configure_splitk<kEpiBias>()) != cudaSuccess) return e;
+  if ((e = configure_splitk<kEpiBiasGelu>()) != cudaSuccess) return e;
+  if ((e = configure_splitk<kEpiLnBias>()) != cudaSuccess) return e;
+  if ((e = configure_splitk<kEpiLnBiasGelu>()) != cudaSuccess) return e;
+  if ((e = configure_splitk<kEpiResidSplit>()) != cudaSuccess) return e;
   return cudaSuccess;
 }
 
@@ -744,6 +951,14 @@ static void launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUten
   const int grid = (int)(tiles < num_sms ? tiles : num_sms);
   launch_dependent(gemm_bf16_kernel<128, EPI>, dim3(grid), dim3(kGemmThreads), SmemPlan<128, EPI>::kSmemBytes, s, 1, pdl,
                    ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag);
+}
+
+template <int EPI>
+static void launch_splitk(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
+                          long M, int N, int K, const EpiParams& ep, int* err_flag, int split, bool pdl, cudaStream_t s) {
+  const long tiles = ((M + kBM - 1) / kBM) * ((N + 127) / 128);
+  launch_dependent(gemm_bf16_splitk_kernel<EPI>, dim3((unsigned)(tiles * split)), dim3(kGemmThreads),
+                   SmemPlan<128, EPI, 1>::kSmemBytes, s, split, pdl, ta, tb, tc, tc2, M, N, K, ep, err_flag, split);
 }
 
 template <int EPI>
@@ -775,6 +990,21 @@ void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtens
     const double r_pair = (double)((t_pair + n_pairs - 1) / n_pairs);
     const double r_small = (double)((t_small + num_sms - 1) / num_sms) * 0.5 * kSmallTilePenalty;
     if (r_small < r_pair) {
+      // so few tiles that half of the SMs or more would idle, and a K range long enough for the
+      // hand-over between the CTAs to pay: split every tile's K range over a cluster of 2 or 4 CTAs
+      const long num_k = (K + kBK - 1) / kBK;
+      const bool may = opt.split_k > 0 && num_k >= opt.split_k;
+      const int split = (may && t_small * 4 <= num_sms && num_k >= 16) ? 4 : (may && t_small * 2 <= num_sms && num_k >= 8) ? 2 : 1;
+      if (split > 1) {
+        switch (epi) {
+          case kEpiBias: launch_splitk<kEpiBias>(ta, tb, tc, tc2, M, N, K, ep, err_flag, split, pdl, s); break;
+          case kEpiBiasGelu: launch_splitk<kEpiBiasGelu>(ta, tb, tc, tc2, M, N, K, ep, err_flag, split, pdl, s); break;
+          case kEpiLnBias: launch_splitk<kEpiLnBias>(ta, tb, tc, tc2, M, N, K, ep, err_flag, split, pdl, s); break;
+          case kEpiLnBiasGelu: launch_splitk<kEpiLnBiasGelu>(ta, tb, tc, tc2, M, N, K, ep, err_flag, split, pdl, s); break;
+          default: launch_splitk<kEpiResidSplit>(ta, tb, tc, tc2, M, N, K, ep, err_flag, split, pdl, s); break;
+        }
+        return;
+      }
       switch (epi) {
         case kEpiBias: launch_one<kEpiBias>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
         case kEpiBiasGelu: launch_one<kEpiBiasGelu>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;

@@ -60,6 +60,8 @@ struct EpiParams {
 struct LaunchOpts {
   int pdl;          // launch with programmatic stream serialization (a kernel's set-up overlaps its predecessor's tail)
   int small_tiles;  // GEMMs too small to fill the CTA pairs run 128 x 128 tiles on single CTAs
+  int split_k;      // ... and, when even those leave half of the SMs idle and K has at least this many 64-wide
+                    // blocks, split each tile's K range over a cluster of CTAs (0: never)
 };
 
 // Offsets (in ints) of the per-call metadata arrays inside one device int buffer.

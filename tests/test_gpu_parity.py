@@ -167,7 +167,7 @@ def enc2_encode(shape, W, audio, lengths):
 # ------------------------------------------------------------------------------ bf16 components
 
 @pytest.mark.parametrize("M,N,K", [(300, 384, 240), (1000, 1536, 512), (129, 256, 64), (4097, 1280, 1280),
-                                   (77, 8, 8)])
+                                   (77, 8, 8), (75, 5120, 1280), (200, 1000, 1024)])   # the last two: K split over a cluster
 @pytest.mark.parametrize("mode", [0, 1])
 def test_tcgen05_gemm_matches_fp64(M, N, K, mode):
     shape = _small("bf16", n_layer=0)
@@ -195,6 +195,13 @@ def _split_planes(x):
     return hi, lo, hi.double().cpu().numpy() + lo.double().cpu().numpy()
 
 
+@pytest.fixture(autouse=True)
+def _split_every_small_gemm(monkeypatch):
+    """Encoders created by the tests of this file split the K range of small GEMMs from 8 K blocks on
+    (the library's default is 64), so that the cluster split is exercised on all three kinds of epilogue."""
+    monkeypatch.setenv("WF_GEMM_SPLIT_K", "8")
+
+
 def _row_stats(x64):
     """[K / 128, M, 2] float32 partial (sum, sum of squares) of every 128 columns."""
     M, K = x64.shape
@@ -203,7 +210,7 @@ def _row_stats(x64):
 
 
 @pytest.mark.parametrize("M,N,K", [(300, 384, 240), (1000, 1536, 512), (129, 256, 64), (4097, 1280, 1280),
-                                   (77, 128, 8), (60, 1280, 5120)])
+                                   (77, 128, 8), (60, 1280, 5120), (775, 1280, 5120), (775, 1280, 1280)])   # the last three: K split over a cluster of 4 / 2 / 2
 def test_tcgen05_residual_gemm_on_split_stream(M, N, K):
     """x <- x + A W^T + bias with x held as two bf16 planes (16 significant bits), and the row
     statistics the epilogue leaves for the LayerNorm that follows."""
@@ -228,7 +235,8 @@ def test_tcgen05_residual_gemm_on_split_stream(M, N, K):
     enc.close()
 
 
-@pytest.mark.parametrize("M,N,K", [(300, 384, 256), (1000, 1536, 512), (129, 256, 128), (4097, 3840, 1280), (77, 8, 128)])
+@pytest.mark.parametrize("M,N,K", [(300, 384, 256), (1000, 1536, 512), (129, 256, 128), (4097, 3840, 1280), (77, 8, 128),
+                                   (100, 3840, 1280), (275, 1280, 1024)])   # the last two: K split over a cluster
 @pytest.mark.parametrize("gelu", [False, True])
 def test_tcgen05_gemm_with_folded_layernorm(M, N, K, gelu):
     """(gelu of) LN(x) W^T + bias computed as rstd (x_hi W'^T - mean s) + c from the bf16 upper plane
