@@ -188,8 +188,10 @@ class Prof {
 // non-empty (kind 0, n_head items each), then one entry for its odd last tile if it has one
 // (kind 1, two heads side by side: ceil(n_head / 2) items), then one int per item naming its entry.
 // *n_items counts the bf16 items.
+// With `num_sms` > 0 and few enough tokens that even one item per (128-row tile, head) gives no more
+// items than SMs, the bf16 list is made of such single-tile items instead (kind 2).
 int build_attn_work(const int* tok, const std::vector<int>& order, bool bf16, int n_head, int* dst, int* n_entries,
-                    int* n_items) {
+                    int* n_items, int num_sms = 0) {
   int nw = 0;
   *n_items = 0;
   if (!bf16) {
@@ -203,6 +205,18 @@ int build_attn_work(const int* tok, const std::vector<int>& order, bool bf16, in
     return 2 * nw;
   }
   int items = 0;
+  long single = 0;
+  for (int i : order) single += (long)((tok[i + 1] - tok[i] + 127) / 128) * n_head;
+  if (num_sms > 0 && single <= num_sms) {
+    for (int i : order)
+      for (int q0 = 0; q0 < tok[i + 1] - tok[i]; q0 += 128) {
+        dst[3 * nw] = i;
+        dst[3 * nw + 1] = (int)((unsigned)q0 | (2u << 30));
+        dst[3 * nw + 2] = items;
+        items += n_head;
+        ++nw;
+      }
+  } else
   for (int i : order) {
     const int n = tok[i + 1] - tok[i];
     for (int q0 = 0; q0 + 128 < n; q0 += 256) {
@@ -298,7 +312,7 @@ wf_status make_plan(wf_encoder* e, const long* len, bool frames_given, int B, Pl
     return hm[ml.tok_off + a + 1] - hm[ml.tok_off + a] > hm[ml.tok_off + b + 1] - hm[ml.tok_off + b];
   });
   int nw = 0, n_items = 0, work_ints = 0;
-  if (build_work) work_ints = build_attn_work(hm + ml.tok_off, order, e->bf16, c.n_head, hm + ml.attn_work, &nw, &n_items);
+  if (build_work) work_ints = build_attn_work(hm + ml.tok_off, order, e->bf16, c.n_head, hm + ml.attn_work, &nw, &n_items, e->num_sms);
   ml.total = ml.attn_work + work_ints;
   p->B = B;
   p->total_samples = samples;
@@ -661,7 +675,7 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
   WF_TRY(dev_alloc_bytes(e, &e->out_stage, mt * d * e->esz));
   WF_TRY(dev_alloc<int>(e, &e->err_flag, 1, true));
   e->meta_cap = 6 * (c.max_batch + 1) + 2 * (int)(c.max_tokens / 16 + c.max_batch) + 6 * c.max_batch + 16 +
-                (e->bf16 ? (int)(c.max_tokens / 256 + 2 * c.max_batch) * c.n_head : 0);
+                (e->bf16 ? (int)(c.max_tokens / 128 + 2 * c.max_batch) * c.n_head : 0);
   for (int i = 0; i < kRing; ++i) {
     WF_TRY(dev_alloc<int>(e, &e->meta_dev[i], e->meta_cap));
     void* hp = nullptr;
@@ -1202,7 +1216,7 @@ wf_status wf_attention(wf_encoder* e, const void* qkv, const int* cu_seqlens, in
   std::vector<int> order(B);
   for (int i = 0; i < B; ++i) order[i] = i;
   int nw = 0, n_items = 0;
-  ml.total = ml.attn_work + build_attn_work(hm, order, e->bf16, e->cfg.n_head, hm + ml.attn_work, &nw, &n_items);
+  ml.total = ml.attn_work + build_attn_work(hm, order, e->bf16, e->cfg.n_head, hm + ml.attn_work, &nw, &n_items, e->num_sms);
   Plan p{};
   p.ml = ml;
   st = ring_upload(e, slot, p, s);

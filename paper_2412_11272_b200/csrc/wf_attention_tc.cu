@@ -83,7 +83,9 @@ struct Item {
 
 // The work list holds (sequence, first query row | kind << 30, first item) triples in launch order;
 // kind 0: 256 consecutive rows (both tiles non-empty), one item per head; kind 1: the odd last
-// tile of a sequence, one item per pair of heads (a last unpaired head runs as a single tile).
+// tile of a sequence, one item per pair of heads (a last unpaired head runs as a single tile);
+// kind 2: one 128-row tile of one head (the planner's choice when that still gives no more items
+// than there are SMs: half the work per CTA, and a lone tile's exponentials run faster).
 // An entry of kind 1 directly follows the other entries of its sequence, so that its K / V tiles
 // are still in the L2 when it runs.  Behind the triples sits one int per item: its entry.
 __device__ __forceinline__ Item load_item(const int* __restrict__ meta, const MetaLayout& ml, int it, int n_head,
@@ -94,9 +96,10 @@ __device__ __forceinline__ Item load_item(const int* __restrict__ meta, const Me
   const int seq = wl[3 * lo], q0k = wl[3 * lo + 1];
   Item w;
   w.q0 = q0k & 0x3FFFFFFF;
-  if ((q0k >> 30) == 0) {
+  const unsigned kind = (unsigned)q0k >> 30;
+  if (kind == 0 || kind == 2) {
     w.head = w.head1 = local;
-    w.two = true;
+    w.two = kind == 0;
     w.split = false;
   } else {
     w.head = 2 * local;

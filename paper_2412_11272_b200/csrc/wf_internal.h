@@ -189,7 +189,8 @@ void launch_layernorm_split(const __nv_bfloat16* x_hi, const __nv_bfloat16* x_lo
                             __nv_bfloat16* out, long M, int d, bool pdl, cudaStream_t s);
 
 // ---- bf16 attention on tcgen05 (wf_attention_tc.cu).  The work list at ml.attn_work holds
-// n_entries triples (sequence, first query row | kind << 30, first item): kind 0 = 256 consecutive
+// n_entries triples (sequence, first query row | kind << 30, first item; kind 2 = one 128-row tile,
+// one item per head, used for small batches): kind 0 = 256 consecutive
 // query rows, one item per head; kind 1 = the odd last 128-row tile of a sequence, one item per
 // pair of heads; behind the triples one int per item names its entry.  n_items is the total.
 cudaError_t attention_bf16_configure();
