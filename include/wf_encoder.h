@@ -146,6 +146,23 @@ wf_status wf_encode_host(wf_encoder *enc, const float *audio_host, const long *l
                          const float *hush_mel, void *hidden_out_host, int *cu_seqlens_out,
                          void *stream);
 
+/* The host-side planner of wf_encode / wf_encode_mel alone: no device, no encoder handle, no CUDA
+ * call.  Row arithmetic of the method (Sec. 4.1.2: 100 log-mel rows per second, the hush segment
+ * appended; Sec. 2.1: two rows per encoder token) and the ragged work lists, with the same
+ * validation and status codes as the encoding calls.
+ *   lengths             host  B sample counts, or frame counts if lengths_are_frames != 0
+ *   tail_samples              raw-audio hush samples that follow every buffer (wf_encode_raw_hush), else 0
+ *   num_sms                   SM count the attention work list is planned for (0: never use single-tile items)
+ *   cu_seqlens_out      host  B+1 token prefix sums (may be NULL)
+ *   totals_out          host  6 values: log-mel frames, rows of the padded-row layout, tokens,
+ *                             front-end tiles, attention work-list entries, attention items (may be NULL)
+ *   work_out, work_cap  host  the attention work list as the kernels read it (may be NULL): WF_F32 pairs
+ *                             (sequence, first query row) per 16 rows; WF_BF16 triples (sequence, first query
+ *                             row | kind << 30, first item) followed by one entry index per item */
+wf_status wf_plan(const wf_config *cfg, const long *lengths, int B, int lengths_are_frames,
+                  long tail_samples, int num_sms, int *cu_seqlens_out, long *totals_out,
+                  int *work_out, int work_cap);
+
 /* Synchronises `stream` and reports WF_ERR_DEVICE_TIMEOUT if any kernel's bounded wait gave
  * up since the last check, WF_ERR_CUDA if the stream is in error, else WF_OK. */
 wf_status wf_check(wf_encoder *enc, void *stream);

@@ -54,7 +54,7 @@ _PER_LAYER = ("ln1_g", "ln1_b", "wq", "bq", "wk", "wv", "bv", "wo", "bo", "ln2_g
 
 EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_raw_hush", "wf_encode_mel", "wf_encode_host", "wf_check",
            "wf_encoder_destroy", "wf_last_error", "wf_profile_enable", "wf_profile_read",
-           "wf_gemm_bf16", "wf_gemm_resid_bf16", "wf_ln_fold", "wf_gemm_ln_bf16", "wf_selftest_wait_timeout", "wf_attention", "wf_cross_kv", "wf_dtw",
+           "wf_plan", "wf_gemm_bf16", "wf_gemm_resid_bf16", "wf_ln_fold", "wf_gemm_ln_bf16", "wf_selftest_wait_timeout", "wf_attention", "wf_cross_kv", "wf_dtw",
            "wf_streams_create", "wf_streams_destroy", "wf_streams_length", "wf_streams_push", "wf_encode_streams", "wf_attention_f32_static",
            "wf_beam_pruner_create", "wf_beam_pruner_step", "wf_beam_pruner_state", "wf_beam_pruner_destroy")
 
@@ -80,6 +80,7 @@ def load_library() -> C.CDLL:
     lib.wf_encoder_destroy.argtypes = [vp]
     lib.wf_last_error.argtypes = [vp]
     lib.wf_last_error.restype = C.c_char_p
+    lib.wf_plan.argtypes = [C.POINTER(wf_config), lp, C.c_int, C.c_int, C.c_long, C.c_int, ip, lp, ip, C.c_int]
     lib.wf_selftest_wait_timeout.argtypes = [vp, C.c_uint, vp]
     lib.wf_profile_enable.argtypes = [vp, C.c_int]
     lib.wf_profile_read.argtypes = [vp, lp, C.POINTER(C.c_double)]
@@ -341,6 +342,27 @@ class Encoder:
         self._check(self.lib.wf_attention(self.handle, qkv.data_ptr(), cu.ctypes.data_as(C.POINTER(C.c_int)),
                                           len(cu) - 1, out.data_ptr(), _stream_ptr(stream)))
         return out
+
+
+def wf_plan(shape, lengths, hush_frames: int, max_batch: int, max_tokens: int, max_samples: int, frames_given=False,
+            tail_samples: int = 0, num_sms: int = 148, n_ctx=None):
+    """The host-side planner alone (no GPU): returns (cu_seqlens, totals dict, attention work list)."""
+    lib = load_library()
+    cfg = wf_config(shape.n_mel, shape.d_model, shape.n_layer, shape.n_head, shape.d_mlp, n_ctx or shape.n_ctx, hush_frames,
+                    1 if shape.dtype == "bf16" else 0, max_batch, max_tokens, max_samples)
+    B = len(lengths)
+    arr, ptr = _longs(lengths)
+    cu = (C.c_int * (B + 1))()
+    totals = (C.c_long * 6)()
+    cap = 8 * (max_tokens // 16 + B + 4) + 4 * (max_tokens // 128 + 2 * B + 2) * max(shape.n_head, 1)
+    work = (C.c_int * cap)()
+    st = lib.wf_plan(C.byref(cfg), ptr, B, 1 if frames_given else 0, tail_samples, num_sms, cu, totals, work, cap)
+    if st != 0:
+        raise WfError(st, "wf_plan rejected the batch")
+    names = ("frames", "padded_rows", "tokens", "front_end_tiles", "attention_entries", "attention_items")
+    t = dict(zip(names, [int(v) for v in totals]))
+    n = (2 * t["attention_entries"]) if shape.dtype != "bf16" else (3 * t["attention_entries"] + t["attention_items"])
+    return np.array(cu[:B + 1]), t, np.array(work[:n])
 
 
 def wf_attention_f32_static(qkv: torch.Tensor, cu_seqlens, d_model: int, out: torch.Tensor, stream=None):

@@ -813,6 +813,39 @@ wf_status wf_encode_host(wf_encoder* e, const float* audio_host, const long* len
   return WF_OK;
 }
 
+wf_status wf_plan(const wf_config* cfg, const long* lengths, int B, int lengths_are_frames, long tail_samples,
+                  int num_sms, int* cu_seqlens_out, long* totals_out, int* work_out, int work_cap) {
+  if (!cfg || B < 0 || tail_samples < 0) return WF_ERR_INVALID_ARG;
+  wf_encoder tmp{};  // the planner reads the configuration only; no CUDA call is made
+  tmp.cfg = *cfg;
+  tmp.bf16 = cfg->dtype == WF_BF16;
+  tmp.num_sms = num_sms;
+  tmp.err[0] = 0;
+  if (B > cfg->max_batch) return WF_ERR_CAPACITY;
+  const size_t cap = 6 * ((size_t)B + 1) + 2 * ((size_t)cfg->max_tokens / 16 + B) + 16 +
+                     ((size_t)cfg->max_tokens / 128 + 2 * (size_t)B + 2) * (size_t)std::max(cfg->n_head, 1) * 2;
+  std::vector<int> hm(cap);
+  Plan p;
+  wf_status st = make_plan(&tmp, lengths, lengths_are_frames != 0, B, &p, hm.data(), false, tail_samples);
+  if (st != WF_OK) return st;
+  if (cu_seqlens_out)
+    for (int i = 0; i <= B; ++i) cu_seqlens_out[i] = hm[p.ml.tok_off + i];
+  if (totals_out) {
+    totals_out[0] = p.total_frames;
+    totals_out[1] = p.total_prows;
+    totals_out[2] = p.total_tokens;
+    totals_out[3] = p.n_fe_tiles;
+    totals_out[4] = p.n_work;
+    totals_out[5] = p.n_attn_items;
+  }
+  if (work_out) {
+    const int n = p.ml.total - p.ml.attn_work;
+    if (n > work_cap) return WF_ERR_CAPACITY;
+    for (int i = 0; i < n; ++i) work_out[i] = hm[p.ml.attn_work + i];
+  }
+  return WF_OK;
+}
+
 wf_status wf_check(wf_encoder* e, void* stream) {
   if (!e) return WF_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
