@@ -8,7 +8,8 @@ one ragged batch.  Audio-seconds count real audio only; tokens include the hush 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
 Under torchrun every rank runs the same workload on its own streams (weak scaling, no
-data-path collective).  ``--impl reference`` times the fp64 CPU oracle on a bounded sample.
+data-path collective); with ``--scaling strong`` the ranks share ONE workload of 64 streams, split by
+cost, and all-gather the packed hidden states after every call.  ``--impl reference`` times the fp64 CPU oracle on a bounded sample.
 """
 from __future__ import annotations
 
@@ -265,17 +266,27 @@ def run_ours(args, rank, world, local_rank):
     hush_np = I.round_to_bf16(I.hush_mel(seed, shape.n_mel))
     hush = torch.as_tensor(hush_np).to(dev)
 
-    # this rank's 64 streams (stream ids continue across ranks: weak scaling, no exchange)
-    streams = np.stack([I.large_stream(seed, s) for s in sharding.rank_stream_ids(rank, N_STREAMS)])
-    max_tokens = int(I.tokens_of([15 * I.SAMPLE_RATE] * N_STREAMS).sum())
-    max_samples = N_STREAMS * 15 * I.SAMPLE_RATE
-    enc = Encoder(shape, W, F, N_STREAMS, max_tokens, max_samples, device=dev)
+    strong = args.scaling == "strong"
+    if strong:
+        # ONE workload of 64 streams split over the ranks by cost (longest-processing-time-first); after
+        # every call the packed hidden states of all 64 streams are gathered on every rank
+        cost = sharding.sequence_cost(I.tokens_of([15 * I.SAMPLE_RATE] * N_STREAMS), shape.d_model, shape.d_mlp, shape.n_layer)
+        parts = sharding.lpt_partition(cost, world)
+        my_ids = parts[rank]
+    else:
+        # this rank's 64 streams (stream ids continue across ranks: weak scaling, no exchange)
+        parts, my_ids = None, sharding.rank_stream_ids(rank, N_STREAMS)
+    n_local = len(my_ids)
+    streams = np.stack([I.large_stream(seed, s) for s in my_ids])
+    max_tokens = int(I.tokens_of([15 * I.SAMPLE_RATE] * n_local).sum())
+    max_samples = n_local * 15 * I.SAMPLE_RATE
+    enc = Encoder(shape, W, F, n_local, max_tokens, max_samples, device=dev)
     audio_host, audio_dev, lengths = {}, {}, {}
     for k in ROUNDS:
         a = np.ascontiguousarray(streams[:, : k * I.SAMPLE_RATE]).reshape(-1)
         audio_host[k] = torch.as_tensor(a).pin_memory()
         audio_dev[k] = audio_host[k].to(dev)
-        lengths[k] = np.full(N_STREAMS, k * I.SAMPLE_RATE, dtype=np.int64)
+        lengths[k] = np.full(n_local, k * I.SAMPLE_RATE, dtype=np.int64)
     out_dev = torch.empty((max_tokens, shape.d_model), dtype=torch.bfloat16, device=dev)
     out_host = torch.empty((max_tokens, shape.d_model), dtype=torch.bfloat16).pin_memory()
 
@@ -285,9 +296,14 @@ def run_ours(args, rank, world, local_rank):
     step_flops = sum(f["encoder"] for f in flops.values())
     step_gemm_flops = sum(f["gemm"] for f in flops.values())
 
+    tokens_all = {k: I.tokens_of([k * I.SAMPLE_RATE] * N_STREAMS) for k in ROUNDS}
+    local_tokens = {k: int(I.tokens_of(lengths[k]).sum()) for k in ROUNDS}
+
     def step():
         for k in ROUNDS:
             enc.wf_encode(audio_dev[k], lengths[k], hush, out=out_dev)
+            if strong and world > 1:
+                sharding.gather_packed(out_dev[: local_tokens[k]], tokens_all[k], parts)
 
     def step_host():
         for k in ROUNDS:
@@ -367,9 +383,12 @@ def run_ours(args, rank, world, local_rank):
         return
     peaks = measured_peaks()
     sec = elapsed_ms / 1e3
-    value = world * args.steps * step_audio_s / sec
+    # whole-job totals: every rank's own streams (weak), or the one workload all ranks share (strong)
+    job_audio_s = step_audio_s * world if not strong else sum(k * N_STREAMS for k in ROUNDS)
+    job_tokens = step_tokens * world if not strong else int(sum(t.sum() for t in tokens_all.values()))
+    value = args.steps * job_audio_s / sec
     tflops = args.steps * step_flops / sec / 1e12            # per GPU
-    per_buffer = [t / N_STREAMS for k in ROUNDS for t in call_ms[k]]
+    per_buffer = [t / n_local for k in ROUNDS for t in call_ms[k]]
     gemm = prof["block_gemm"]
     gemm_flops_per_launch = args.steps * step_gemm_flops / max(gemm["launches"], 1)
     gemm_tflops = gemm_flops_per_launch / (gemm["ms"] / max(gemm["launches"], 1) / 1e3) / 1e12 if gemm["ms"] > 0 else None
@@ -377,19 +396,20 @@ def run_ours(args, rank, world, local_rank):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "streams_per_gpu": N_STREAMS, "calls_per_step": len(ROUNDS),
+        "scaling": "strong" if strong else "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "streams_per_gpu": n_local, "calls_per_step": len(ROUNDS),
                    "tokens_per_step": step_tokens, "audio_seconds_per_step": step_audio_s,
                    "l2": "activations and weights of every call exceed the 126 MB L2 (1.26 GB of weights per call)",
-                   "parallelism": f"dp{world} (independent streams per rank)",
+                   "parallelism": (f"dp{world} (one batch of {N_STREAMS} streams split by cost, packed outputs all-gathered)" if strong
+                                   else f"dp{world} (independent streams per rank)"),
                    "timed_region": "K steps of 15 wf_encode calls back to back, no event or profiling call inside"},
-        "tokens_per_sec": world * args.steps * step_tokens / sec,
+        "tokens_per_sec": args.steps * job_tokens / sec,
         "algorithmic_tflops_per_gpu": tflops,
         "frac_bf16_peak": {"burst": tflops / peaks["bf16_burst"], "sustained": tflops / peaks["bf16_sustained"],
                            "of": peaks["source"]},
         "p50_ms_per_buffer": statistics.median(per_buffer), "p90_ms_per_buffer": float(np.percentile(per_buffer, 90)),
         "clocks": clocks,
-        "e2e": {"value": world * args.steps * step_audio_s / (e2e_ms / 1e3), "unit": UNIT,
+        "e2e": {"value": args.steps * job_audio_s / (e2e_ms / 1e3), "unit": UNIT,
                 "h2d_bytes_per_step": int(sum(audio_host[k].numel() * 4 for k in ROUNDS)),
                 "d2h_bytes_per_step": int(step_tokens * shape.d_model * 2)},
         "gpu_launches": int(launches),
@@ -431,6 +451,8 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak: every rank encodes its own 64 streams; strong: one workload of 64 streams split over the ranks")
     ap.add_argument("--no-other-configs", action="store_true", help="skip the smaller configurations' section")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

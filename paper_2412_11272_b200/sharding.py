@@ -59,6 +59,34 @@ def reassemble_packed(shards, parts, tokens) -> np.ndarray:
     return out
 
 
+def gather_packed(local: torch.Tensor, tokens, parts) -> torch.Tensor:
+    """The collective behind a strong-scaling split: every rank contributes the packed hidden
+    states of its own sequences (`local`, [sum of its tokens, d], on the device of the process
+    group's backend) and receives the whole batch's packed rows in the original sequence order.
+    One all-gather of shards padded to the largest shard (NCCL over NVLink on GPUs, gloo on CPU);
+    nothing else crosses ranks.  `parts[r]` lists rank r's sequences, `tokens` every sequence's
+    token count.  Without a process group (or with one rank) it returns `local` reordered."""
+    tokens = np.asarray(tokens, dtype=np.int64)
+    cu = np.concatenate([[0], np.cumsum(tokens)])
+    world = dist.get_world_size() if dist.is_available() and dist.is_initialized() else 1
+    rows = [int(tokens[list(p)].sum()) for p in parts]
+    if world == 1:
+        shards = [local]
+    else:
+        pad = max(rows)
+        mine = torch.zeros((pad, local.shape[1]), dtype=local.dtype, device=local.device)
+        mine[: local.shape[0]] = local
+        bufs = [torch.empty_like(mine) for _ in range(world)]
+        dist.all_gather(bufs, mine)
+        shards = [b[:n] for b, n in zip(bufs, rows)]
+    out = torch.empty((int(cu[-1]), local.shape[1]), dtype=local.dtype, device=local.device)
+    for shard, part in zip(shards, parts):
+        lc = rank_cu_seqlens(tokens, part)
+        for j, i in enumerate(part):
+            out[cu[i]:cu[i + 1]] = shard[lc[j]:lc[j + 1]]
+    return out
+
+
 def max_over_ranks(value: float, device="cpu") -> float:
     """The slowest rank's time: what a multi-GPU throughput has to be computed from."""
     if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:

@@ -40,6 +40,9 @@ def _worker(rank, world, port, out_dir):
         whole = sharding.reassemble_packed(shards, all_parts, tokens)
         expect = np.concatenate([np.stack([np.full(t, i), np.arange(t)], axis=1) for i, t in enumerate(tokens)])
         reassembled = float(np.array_equal(whole, expect))
+        # the same through the collective (one all-gather of padded shards)
+        gathered_rows = sharding.gather_packed(torch.as_tensor(rows), tokens, all_parts)
+        reassembled *= float(np.array_equal(gathered_rows.numpy(), expect))
         np.save(os.path.join(out_dir, f"r{rank}.npy"),
                 np.array([slowest, float(sorted(sum(gathered, [])) == list(range(4 * world))),
                           float(sorted(sum(all_parts, [])) == list(range(64))), max(loads) / (sum(loads) / world),
