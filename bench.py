@@ -181,7 +181,7 @@ def time_calls(fn, iters, warmup=5):
     return t[len(t) // 2], t[int(len(t) * 0.9)]
 
 
-def other_configs(dev, large_enc, large_audio, large_hush):
+def other_configs(dev, large_enc, large_audio, large_hush, large_ref):
     """The smaller named configurations, each timed per call (device-resident inputs) and checked
     on one whole sequence against the oracle: latency-bound cases (tiny, base, one 15 s large-v3
     buffer), the 64-buffer small-shaped batch, and the medium-shaped batch once padded to 30 s and
@@ -244,8 +244,11 @@ def other_configs(dev, large_enc, large_audio, large_hush):
     L = SAMPLE_SECONDS * I.SAMPLE_RATE
     one = large_audio[:L].contiguous()
     p50, p90 = time_calls(lambda: large_enc.wf_encode(one, [L], large_hush), 50)
+    res, _ = large_enc.wf_encode(one, [L], large_hush)
+    large_enc.wf_check()
     out["large_single_15s_buffer"] = {"dtype": "bf16", "buffers": 1, "tokens": int(I.tokens_of([L])[0]), "ms_per_call": p50,
-                                      "p90_ms_per_call": p90, "audio_s_per_s": SAMPLE_SECONDS / p50 * 1e3}
+                                      "p90_ms_per_call": p90, "audio_s_per_s": SAMPLE_SECONDS / p50 * 1e3,
+                                      "parity": parity_of(res.float().cpu().numpy().astype(np.float64), large_ref)}
     return out
 
 
@@ -440,7 +443,7 @@ def run_ours(args, rank, world, local_rank):
                                 "sample": f"stream 0's first {SAMPLE_SECONDS} s + 50 hush frames (775 tokens), all 32 layers, {dt:.1f} s of CPU time"}
         if not args.no_other_configs:
             del W
-            line["other_configs"] = other_configs(dev, enc, audio_dev[SAMPLE_SECONDS], hush)
+            line["other_configs"] = other_configs(dev, enc, audio_dev[SAMPLE_SECONDS], hush, ref)
     enc.close()
     print(json.dumps(line), flush=True)
 

@@ -188,8 +188,12 @@ __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtenso
     }
   } else {
     // bf16: 64 columns = 128 bytes per row and piece
-    bool valid = true;
-    if (EPI == kEpiConv1) valid = row < M && ep.row_valid[row] != 0;
+    // Rows at or beyond M that the last tile still stores (outputs are capacity-sized) are written as
+    // zeros, never as whatever the accumulator holds for them: the attention kernel multiplies the
+    // value rows behind a sequence's end by probabilities that are exactly zero, which only gives
+    // zero if those rows are finite.
+    bool valid = row < M;
+    if (EPI == kEpiConv1) valid = valid && ep.row_valid[row] != 0;
     float2 nrm = make_float2(0.f, 0.f);
     if (epi_is_ln(EPI)) nrm = row_norm(ep, row, M, K);
 #pragma unroll 1
@@ -205,7 +209,7 @@ __device__ __forceinline__ void epilogue_tile(const EpiParams& ep, const CUtenso
         tmem_ld_wait();
         if (ps.n > 0) add_partials(ps, quarter * 32 + lane, c * 64 + hf * 32, a32);
         bias_act32<EPI>(ep, n0 + c * 64 + hf * 32, N, a32, v, nrm);
-        if (EPI == kEpiConv1 && !valid) {
+        if (!valid) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = 0.f;
         }
@@ -302,6 +306,10 @@ __device__ __forceinline__ bool epilogue_tile_split(const EpiParams& ep, const C
         tmem_ld_wait();
         if (ps.n > 0) add_partials(ps, quarter * 32 + lane, c * 64 + hf * 32, a32);
         bias_act32<kEpiResidSplit>(ep, n0 + c * 64 + hf * 32, N, a32, v, make_float2(0.f, 0.f));
+        if (row >= M) {  // a row beyond the matrix inside a stored piece keeps its old value
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = 0.f;
+        }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const uint32_t a = buf + lane * 128 + (((hf * 4 + j) ^ (lane & 7)) << 4);

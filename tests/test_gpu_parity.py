@@ -447,6 +447,27 @@ def test_bf16_small_ragged_matches_oracle():
     enc.close()
 
 
+def test_bf16_deep_encoder_with_spare_capacity():
+    """Many layers on an encoder sized far beyond the batch: the rows between the batch's last token and
+    the end of the last stored tile exist in memory and pass through every layer.  They must stay
+    finite (they are written as zeros): the attention kernel multiplies the rows behind a sequence's
+    end by zero probabilities, and anything non-finite there would spoil the last sequence."""
+    shape = _small("bf16", d_model=256, n_head=4, d_mlp=1024, n_layer=24)
+    W = I.encoder_weights(13, shape)
+    batch = I.batch_from_lengths(13, [160 * 150, 160 * 611])          # 100 + 331 tokens: 431 = 3 x 128 + 47
+    hush = I.round_to_bf16(I.hush_mel(13, shape.n_mel))
+    enc = make_encoder(shape, W, 16, 8192, 16 * 160 * 1500)
+    for _ in range(2):                                                   # the second call finds the first call's rows
+        out, cu = enc.wf_encode(_dev(batch.audio), batch.lengths, _dev(hush))
+        enc.wf_check()
+        got = to_np(out)
+        assert np.isfinite(got).all()
+        refs = oracle_hidden(batch, shape, W, hush)
+        for i, ref in refs.items():
+            _check_bf16(got[cu[i]:cu[i + 1]], ref)
+    enc.close()
+
+
 def test_bf16_many_minimal_buffers():
     """400 buffers, most of them the shortest the front end accepts (401 samples: 2 frames + hush =
     26 tokens), some a little longer: work lists, tile maps and metadata at a high sequence count."""
