@@ -38,7 +38,7 @@ ROUNDS = list(range(1, 16))
 # from one ncu capture of the current kernels at M = 16384; the traffic grows in proportion to M
 # (activations dominate, weights are read once per launch), so it is scaled per token to the mean
 # launch of the benchmark.  Set to None whenever a GEMM kernel changes, until re-captured.
-GEMM_DRAM_BYTES_M16384 = (127.4e6, 160.4e6, 173.5e6, 367.6e6)
+GEMM_DRAM_BYTES_M16384 = (127.1e6, 160.9e6, 172.9e6, 368.5e6)
 TRAFFIC_NOTE = "DRAM bytes per launch (mean over the four GEMM shapes), scaled per token from the M = 16384 ncu capture"
 SAMPLE_SECONDS = 15         # the CPU oracle is timed on stream 0's full 15 s window (775 tokens)
 
