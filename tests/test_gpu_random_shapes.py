@@ -108,3 +108,33 @@ def test_encode_random_batches_repeat_and_are_batch_invariant(enc):
         solo = enc.wf_encode(audio[:int(lens[0])].contiguous(), lens[:1], hush)[0]     # sequence 0 alone
         assert float((solo.float() - outs[0][:solo.shape[0]].float()).abs().max()) < 0.1, list(lens)
     enc.wf_check()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_spare_capacity_gives_the_same_bits_as_an_exact_fit(dtype):
+    """One deep encoder sized far beyond its batches, fed batches of very different sizes one after
+    the other, against encoders created to fit each batch exactly: kernel choices depend on the
+    batch, not on the capacity, so every bit must agree -- whatever earlier calls left in the
+    workspace rows behind the batch's last token."""
+    n_layer = 16 if dtype == "bf16" else 3
+    shape = I.EncoderShape("cap", 80, 128, n_layer, 2, 256, dtype, n_ctx=1600)
+    W = I.encoder_weights(5, shape)
+    hush_np = I.hush_mel(5, 80)
+    hush = torch.as_tensor(I.round_to_bf16(hush_np) if dtype == "bf16" else hush_np).cuda()
+    big = make_encoder(shape, W, 32, 20000, 32 * 160 * 1500)
+    rng = np.random.default_rng(103)
+    for case in range(8):
+        B = int(rng.choice([1, 2, 17, 32]))
+        lens = np.array([160 * int(rng.integers(3, 1200 if case % 2 else 60)) + int(rng.integers(0, 160)) for _ in range(B)])
+        lens = lens[: max(1, min(B, int(19000 // max(1, int(I.tokens_of(lens).max())))))]      # stay inside the big encoder's tokens
+        batch = I.batch_from_lengths(200 + case, lens)
+        audio = torch.as_tensor(batch.audio).cuda()
+        got, cu = big.wf_encode(audio, batch.lengths, hush)
+        big.wf_check()
+        fit = make_encoder(shape, W, len(lens), int(cu[-1]), int(batch.lengths.sum()))
+        want, cu2 = fit.wf_encode(audio, batch.lengths, hush)
+        fit.wf_check()
+        assert list(cu) == list(cu2) and bool(torch.isfinite(got.float()).all())
+        assert torch.equal(got, want), (case, list(lens))
+        fit.close()
+    big.close()
