@@ -291,7 +291,7 @@ def run_ours(args, rank, world, local_rank):
         audio_dev[k] = audio_host[k].to(dev)
         lengths[k] = np.full(n_local, k * I.SAMPLE_RATE, dtype=np.int64)
     out_dev = torch.empty((max_tokens, shape.d_model), dtype=torch.bfloat16, device=dev)
-    out_host = torch.empty((max_tokens, shape.d_model), dtype=torch.bfloat16).pin_memory()
+    out_host = [torch.empty((max_tokens, shape.d_model), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
 
     flops = {k: I.algorithmic_flops(shape, lengths[k]) for k in ROUNDS}
     step_audio_s = sum(f["audio_seconds"] for f in flops.values())
@@ -309,8 +309,16 @@ def run_ours(args, rank, world, local_rank):
                 sharding.gather_packed(out_dev[: local_tokens[k]], tokens_all[k], parts)
 
     def step_host():
-        for k in ROUNDS:
-            enc.wf_encode_host(audio_host[k], lengths[k], hush, out_host)
+        # host buffers in, host buffers out, the way a streaming server calls it: the next call is issued
+        # while the previous one's result is still on its way to the host; every result of the step has
+        # arrived before the step ends
+        prev = None
+        for i, k in enumerate(ROUNDS):
+            ticket, _ = enc.wf_encode_host_async(audio_host[k], lengths[k], hush, out_host[i & 1])
+            if prev is not None:
+                enc.wf_encode_host_wait(prev)
+            prev = ticket
+        enc.wf_encode_host_wait(prev)
 
     def barrier():
         sharding.barrier()

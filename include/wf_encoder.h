@@ -146,6 +146,19 @@ wf_status wf_encode_host(wf_encoder *enc, const float *audio_host, const long *l
                          const float *hush_mel, void *hidden_out_host, int *cu_seqlens_out,
                          void *stream);
 
+/* The same without the wait, for a caller that encodes buffer after buffer (every round of the
+ * streaming pipeline re-encodes the stream's buffer, Sec. 4.3.2): the call returns once its work
+ * is enqueued, and the library's two sets of staging buffers let the host-to-device copy of one
+ * call and the device-to-host copy of the previous one run (on two streams of the library's own)
+ * under the kernels in between.  hidden_out_host holds the result, and audio_host may be reused,
+ * once wf_encode_host_wait(ticket) has returned; pass pinned memory, and do not reuse an output
+ * buffer before its ticket has been waited for.  At most two calls are in flight: a third call
+ * first waits for the oldest.  cu_seqlens_out is written before the call returns. */
+wf_status wf_encode_host_async(wf_encoder *enc, const float *audio_host, const long *lengths, int B,
+                               const float *hush_mel, void *hidden_out_host, int *cu_seqlens_out,
+                               void *stream, long *ticket_out);
+wf_status wf_encode_host_wait(wf_encoder *enc, long ticket);
+
 /* The host-side planner of wf_encode / wf_encode_mel alone: no device, no encoder handle, no CUDA
  * call.  Row arithmetic of the method (Sec. 4.1.2: 100 log-mel rows per second, the hush segment
  * appended; Sec. 2.1: two rows per encoder token) and the ragged work lists, with the same

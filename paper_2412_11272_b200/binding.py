@@ -52,7 +52,7 @@ class wf_weights(C.Structure):
 _PER_LAYER = ("ln1_g", "ln1_b", "wq", "bq", "wk", "wv", "bv", "wo", "bo", "ln2_g", "ln2_b",
               "w1", "b1", "w2", "b2")
 
-EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_raw_hush", "wf_encode_mel", "wf_encode_host", "wf_check",
+EXPORTS = ("wf_encoder_create", "wf_logmel", "wf_encode", "wf_encode_raw_hush", "wf_encode_mel", "wf_encode_host", "wf_encode_host_async", "wf_encode_host_wait", "wf_check",
            "wf_encoder_destroy", "wf_last_error", "wf_profile_enable", "wf_profile_read",
            "wf_plan", "wf_gemm_bf16", "wf_gemm_resid_bf16", "wf_ln_fold", "wf_gemm_ln_bf16", "wf_selftest_wait_timeout", "wf_attention", "wf_cross_kv", "wf_dtw",
            "wf_streams_create", "wf_streams_destroy", "wf_streams_length", "wf_streams_push", "wf_encode_streams", "wf_attention_f32_static",
@@ -76,6 +76,8 @@ def load_library() -> C.CDLL:
     lib.wf_encode_mel.argtypes = [vp, vp, lp, C.c_int, vp, vp, ip, vp]
     lib.wf_encode_raw_hush.argtypes = [vp, vp, lp, C.c_int, vp, C.c_int, vp, ip, vp]
     lib.wf_encode_host.argtypes = [vp, vp, lp, C.c_int, vp, vp, ip, vp]
+    lib.wf_encode_host_async.argtypes = [vp, vp, lp, C.c_int, vp, vp, ip, vp, lp]
+    lib.wf_encode_host_wait.argtypes = [vp, C.c_long]
     lib.wf_check.argtypes = [vp, vp]
     lib.wf_encoder_destroy.argtypes = [vp]
     lib.wf_last_error.argtypes = [vp]
@@ -253,6 +255,22 @@ class Encoder:
                                             out_host.data_ptr(), cu.ctypes.data_as(C.POINTER(C.c_int)),
                                             _stream_ptr(stream)))
         return out_host, cu
+
+    def wf_encode_host_async(self, audio_host: torch.Tensor, lengths, hush_mel, out_host: torch.Tensor, stream=None):
+        """As wf_encode_host without the wait: returns (ticket, cu_seqlens); out_host is valid after
+        wf_encode_host_wait(ticket)."""
+        arr, ptr = _longs(lengths)
+        B = len(arr)
+        cu = np.zeros(B + 1, dtype=np.int32)
+        ticket = C.c_long(0)
+        self._check(self.lib.wf_encode_host_async(self.handle, audio_host.data_ptr(), ptr, B,
+                                                  hush_mel.data_ptr() if hush_mel is not None else None,
+                                                  out_host.data_ptr(), cu.ctypes.data_as(C.POINTER(C.c_int)),
+                                                  _stream_ptr(stream), C.byref(ticket)))
+        return int(ticket.value), cu
+
+    def wf_encode_host_wait(self, ticket: int):
+        self._check(self.lib.wf_encode_host_wait(self.handle, ticket))
 
     def wf_check(self, stream=None):
         self._check(self.lib.wf_check(self.handle, _stream_ptr(stream)))

@@ -66,8 +66,14 @@ struct wf_encoder {
   float2* stats;            // bf16 path: [d_model / 128][max_tokens] row partial (sum, sum of squares) of x
   void *qkv, *attn, *fc1;
   LaunchOpts opt;
-  float* audio_stage;
-  void* out_stage;
+  // host-buffer calls: two sets of staging buffers, so that the copies of one call overlap the
+  // kernels of its neighbours (copies run on two streams of the library's own)
+  float* audio_stage[2];
+  void* out_stage[2];
+  cudaStream_t copy_in, copy_out;
+  cudaEvent_t host_ev_in[2], host_ev_comp[2], host_ev_out[2];
+  bool host_used[2];
+  long host_calls;
   int* err_flag;
 
   int meta_cap;
@@ -554,6 +560,9 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
   e->prof_used = 0;
   e->ring_pos = 0;
   for (int i = 0; i < kRing; ++i) { e->meta_used[i] = false; e->meta_dev[i] = nullptr; e->meta_host[i] = nullptr; e->meta_ev[i] = nullptr; }
+  e->copy_in = e->copy_out = nullptr;
+  e->host_calls = 0;
+  for (int i = 0; i < 2; ++i) { e->host_used[i] = false; e->host_ev_in[i] = e->host_ev_comp[i] = e->host_ev_out[i] = nullptr; }
   *out = e;  // returned even on failure so that the caller can read the message, then destroy
   const wf_config& c = e->cfg;
   if (c.n_mel <= 0 || c.n_mel % 8 || c.n_mel > 128 || c.d_model <= 0 || c.d_model % 128 || c.d_model > 1280 ||
@@ -671,8 +680,15 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
   WF_TRY(dev_alloc_bytes(e, &e->qkv, mt * 3 * d * e->esz, true));
   WF_TRY(dev_alloc_bytes(e, &e->attn, mt * d * e->esz, true));
   WF_TRY(dev_alloc_bytes(e, &e->fc1, mt * F * e->esz, true));
-  WF_TRY(dev_alloc<float>(e, &e->audio_stage, (size_t)c.max_samples));
-  WF_TRY(dev_alloc_bytes(e, &e->out_stage, mt * d * e->esz));
+  for (int i = 0; i < 2; ++i) {
+    WF_TRY(dev_alloc<float>(e, &e->audio_stage[i], (size_t)c.max_samples));
+    WF_TRY(dev_alloc_bytes(e, &e->out_stage[i], mt * d * e->esz));
+    WF_CUDA(e, cudaEventCreateWithFlags(&e->host_ev_in[i], cudaEventDisableTiming));
+    WF_CUDA(e, cudaEventCreateWithFlags(&e->host_ev_comp[i], cudaEventDisableTiming));
+    WF_CUDA(e, cudaEventCreateWithFlags(&e->host_ev_out[i], cudaEventDisableTiming));
+  }
+  WF_CUDA(e, cudaStreamCreateWithFlags(&e->copy_in, cudaStreamNonBlocking));
+  WF_CUDA(e, cudaStreamCreateWithFlags(&e->copy_out, cudaStreamNonBlocking));
   WF_TRY(dev_alloc<int>(e, &e->err_flag, 1, true));
   e->meta_cap = 6 * (c.max_batch + 1) + 2 * (int)(c.max_tokens / 16 + c.max_batch) + 6 * c.max_batch + 16 +
                 (e->bf16 ? (int)(c.max_tokens / 128 + 2 * c.max_batch) * c.n_head : 0);
@@ -724,6 +740,13 @@ wf_status wf_encoder_destroy(wf_encoder* e) {
   for (int i = 0; i < kRing; ++i)
     if (e->meta_ev[i]) cudaEventDestroy(e->meta_ev[i]);
   for (auto& pe : e->prof) { cudaEventDestroy(pe.a); cudaEventDestroy(pe.b); }
+  for (int i = 0; i < 2; ++i) {
+    if (e->host_ev_in[i]) cudaEventDestroy(e->host_ev_in[i]);
+    if (e->host_ev_comp[i]) cudaEventDestroy(e->host_ev_comp[i]);
+    if (e->host_ev_out[i]) cudaEventDestroy(e->host_ev_out[i]);
+  }
+  if (e->copy_in) cudaStreamDestroy(e->copy_in);
+  if (e->copy_out) cudaStreamDestroy(e->copy_out);
   delete e;
   return WF_OK;
 }
@@ -790,11 +813,12 @@ wf_status wf_encode_mel(wf_encoder* e, const float* mel, const long* frames, int
   return encode_impl(e, nullptr, mel, frames, B, hush_mel, hidden_out, cu_seqlens_out, (cudaStream_t)stream);
 }
 
-wf_status wf_encode_host(wf_encoder* e, const float* audio_host, const long* lengths, int B,
-                         const float* hush_mel, void* hidden_out_host, int* cu_seqlens_out, void* stream) {
+wf_status wf_encode_host_async(wf_encoder* e, const float* audio_host, const long* lengths, int B,
+                               const float* hush_mel, void* hidden_out_host, int* cu_seqlens_out, void* stream,
+                               long* ticket_out) {
   if (!e) return WF_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  if (B < 0 || (B > 0 && (!audio_host || !lengths || !hidden_out_host)))
+  if (B < 0 || !ticket_out || (B > 0 && (!audio_host || !lengths || !hidden_out_host)))
     return fail(e, WF_ERR_INVALID_ARG, "NULL input or output");
   long total = 0;
   for (int i = 0; i < B; ++i) {
@@ -802,15 +826,41 @@ wf_status wf_encode_host(wf_encoder* e, const float* audio_host, const long* len
     total += lengths[i];
     if (total > e->cfg.max_samples) return fail(e, WF_ERR_CAPACITY, "more than max_samples=%ld samples", e->cfg.max_samples);
   }
-  if (total > 0) WF_CUDA(e, cudaMemcpyAsync(e->audio_stage, audio_host, (size_t)total * sizeof(float), cudaMemcpyHostToDevice, s));
+  const int slot = (int)(e->host_calls & 1);
+  // the call that used this slot two calls ago has delivered its result (and so finished its kernels)
+  if (e->host_used[slot]) WF_CUDA(e, cudaEventSynchronize(e->host_ev_out[slot]));
+  if (total > 0)
+    WF_CUDA(e, cudaMemcpyAsync(e->audio_stage[slot], audio_host, (size_t)total * sizeof(float), cudaMemcpyHostToDevice, e->copy_in));
+  WF_CUDA(e, cudaEventRecord(e->host_ev_in[slot], e->copy_in));
+  WF_CUDA(e, cudaStreamWaitEvent(s, e->host_ev_in[slot], 0));
   std::vector<int> cu(B + 1, 0);
-  wf_status st = encode_impl(e, e->audio_stage, nullptr, lengths, B, hush_mel, e->out_stage, cu.data(), s);
+  wf_status st = encode_impl(e, e->audio_stage[slot], nullptr, lengths, B, hush_mel, e->out_stage[slot], cu.data(), s);
   if (st != WF_OK) return st;
   if (cu_seqlens_out) std::memcpy(cu_seqlens_out, cu.data(), (size_t)(B + 1) * sizeof(int));
-  size_t bytes = (size_t)cu[B] * e->cfg.d_model * e->esz;
-  if (bytes) WF_CUDA(e, cudaMemcpyAsync(hidden_out_host, e->out_stage, bytes, cudaMemcpyDeviceToHost, s));
-  WF_CUDA(e, cudaStreamSynchronize(s));
+  WF_CUDA(e, cudaEventRecord(e->host_ev_comp[slot], s));
+  WF_CUDA(e, cudaStreamWaitEvent(e->copy_out, e->host_ev_comp[slot], 0));
+  const size_t bytes = (size_t)cu[B] * e->cfg.d_model * e->esz;
+  if (bytes) WF_CUDA(e, cudaMemcpyAsync(hidden_out_host, e->out_stage[slot], bytes, cudaMemcpyDeviceToHost, e->copy_out));
+  WF_CUDA(e, cudaEventRecord(e->host_ev_out[slot], e->copy_out));
+  e->host_used[slot] = true;
+  *ticket_out = e->host_calls++;
   return WF_OK;
+}
+
+wf_status wf_encode_host_wait(wf_encoder* e, long ticket) {
+  if (!e) return WF_ERR_INVALID_ARG;
+  if (ticket < 0 || ticket >= e->host_calls) return fail(e, WF_ERR_INVALID_ARG, "unknown ticket %ld", ticket);
+  if (ticket < e->host_calls - 2) return WF_OK;  // its slot has been reused, which waited for it
+  WF_CUDA(e, cudaEventSynchronize(e->host_ev_out[ticket & 1]));
+  return WF_OK;
+}
+
+wf_status wf_encode_host(wf_encoder* e, const float* audio_host, const long* lengths, int B,
+                         const float* hush_mel, void* hidden_out_host, int* cu_seqlens_out, void* stream) {
+  long ticket = 0;
+  wf_status st = wf_encode_host_async(e, audio_host, lengths, B, hush_mel, hidden_out_host, cu_seqlens_out, stream, &ticket);
+  if (st != WF_OK) return st;
+  return wf_encode_host_wait(e, ticket);
 }
 
 wf_status wf_plan(const wf_config* cfg, const long* lengths, int B, int lengths_are_frames, long tail_samples,

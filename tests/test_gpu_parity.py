@@ -524,6 +524,31 @@ def test_bf16_base_config_matches_oracle():
     o_host = torch.empty((M, shape.d_model), dtype=torch.bfloat16).pin_memory()
     enc.wf_encode_host(a_host, batch.lengths, _dev(hush), o_host)
     assert torch.equal(o_host, out.cpu())
+    # and so does the pipelined form: seven calls on sub-batches of different sizes, in flight two at a
+    # time, each compared (after its own ticket) with the synchronous call on the same sub-batch
+    subs = [(0, 16), (3, 9), (0, 1), (5, 16), (15, 16), (2, 4), (0, 16)]
+    offs = np.concatenate([[0], np.cumsum(batch.lengths)])
+    audio_h = [torch.as_tensor(batch.audio[offs[lo]:offs[hi]].copy()).pin_memory() for lo, hi in subs]
+    want = []
+    for (lo, hi), a_h in zip(subs, audio_h):
+        w = torch.empty((int(cu[hi] - cu[lo]), shape.d_model), dtype=torch.bfloat16).pin_memory()
+        enc.wf_encode_host(a_h, batch.lengths[lo:hi], _dev(hush), w)
+        want.append(w.clone())
+    assert torch.equal(want[0], out.cpu())
+    pending = []
+    for j, (lo, hi) in enumerate(subs):
+        o_h = torch.full((int(cu[hi] - cu[lo]), shape.d_model), float("nan"), dtype=torch.bfloat16).pin_memory()
+        ticket, cu_sub = enc.wf_encode_host_async(audio_h[j], batch.lengths[lo:hi], _dev(hush), o_h)
+        assert list(cu_sub) == list(cu[lo:hi + 1] - cu[lo])
+        pending.append((ticket, j, o_h))
+        if len(pending) > 2:
+            t, i, o = pending.pop(0)
+            enc.wf_encode_host_wait(t)
+            assert torch.equal(o, want[i]), subs[i]
+    for t, i, o in pending:
+        enc.wf_encode_host_wait(t)
+        assert torch.equal(o, want[i]), subs[i]
+    enc.wf_check()
     enc.close()
 
 
