@@ -85,12 +85,14 @@ typedef struct {
  * the stated capacities.  Synchronises `stream` before returning.  Fails with
  * WF_ERR_UNSUPPORTED_ARCH on a device that is not compute capability 10.x.
  * (Operation: the encoder of Sec. 1.1 / Sec. 2.3; weights are caller-provided.)
- * Three tuning switches of the WF_BF16 path are read from the environment here and kept in the
+ * Four tuning switches of the WF_BF16 path are read from the environment here and kept in the
  * handle (a later create with another environment does not change this one):
  *   WF_PDL=0               launch kernels plainly instead of with programmatic stream
  *                          serialization (on by default: a kernel's set-up overlaps the tail of
  *                          the kernel before it);
  *   WF_GEMM_SMALL_TILES=0  never use 128 x 128 single-CTA tiles for small GEMMs;
+ *   WF_GEMM_TILE=1|2|3     force 256 x 256 CTA-pair tiles, 128 x 128 or 128 x 256 single-CTA tiles for the
+ *                          block GEMMs instead of letting the launcher choose by the problem's size;
  *   WF_GEMM_SPLIT_K=n      split the K range of a GEMM with few tiles over a cluster of CTAs when K
  *                          has at least n blocks of 64 (default 64; 0 = never).
  * None of them changes what is computed beyond float32 rounding order (which is fixed for a

@@ -596,6 +596,8 @@ wf_status wf_encoder_create(const wf_config* cfg, const wf_weights* w, void* str
     e->opt.pdl = !(pdl_env != nullptr && pdl_env[0] == '0');
     const char* small_env = getenv("WF_GEMM_SMALL_TILES");
     e->opt.small_tiles = !(small_env != nullptr && small_env[0] == '0');
+    const char* tile_env = getenv("WF_GEMM_TILE");
+    e->opt.tile = tile_env != nullptr ? atoi(tile_env) : 0;
     const char* split_env = getenv("WF_GEMM_SPLIT_K");
     e->opt.split_k = split_env != nullptr ? atoi(split_env) : 64;
   }

@@ -365,8 +365,8 @@ __device__ __forceinline__ void drain_stages(uint32_t full_bar0, int stages, uin
   }
 }
 
-// Single-CTA kernel, 128 x 128 tiles: the small-M regime, where 256 x 256 tiles would leave most
-// CTA pairs idle.  tmap_c is the bf16 output map, or x_hi's (with tmap_c2 = x_lo's) for kEpiResidSplit.
+// Single-CTA kernel, 128 x 128 or 128 x 256 tiles: the small-M regime, where 256 x 256 tiles would
+// leave most CTA pairs idle.  tmap_c is the bf16 output map, or x_hi's (with tmap_c2 = x_lo's) for kEpiResidSplit.
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
     const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -435,6 +435,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_bf16_kernel(
           const int e = kb * kBK;
           tma_load_2d(sa, &tmap_a, e % a_cols, m0 + e / a_cols, full_bar(stage));
           tma_load_2d(sa + Cfg::kABytes, &tmap_b, kb * kBK, n0, full_bar(stage));
+          if (BN == 256)  // the W map's box has 128 rows: the second half of a 256-wide tile
+            tma_load_2d(sa + Cfg::kABytes + 128 * kBK * 2, &tmap_b, kb * kBK, n0 + 128, full_bar(stage));
           armed |= 1u << stage;
           armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
           if (++stage == Cfg::kStages) { stage = 0; phase ^= 1u; }
@@ -910,8 +912,11 @@ bool make_tmap_out(const TmaApi& api, CUtensorMap* m, const void* base, int elem
 
 template <int EPI>
 static cudaError_t configure_one() {
-  return cudaFuncSetAttribute(gemm_bf16_kernel<128, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              SmemPlan<128, EPI>::kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel<128, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       SmemPlan<128, EPI>::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_bf16_kernel<256, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              SmemPlan<256, EPI>::kSmemBytes);
 }
 
 template <int EPI>
@@ -951,13 +956,13 @@ cudaError_t gemm_bf16_configure() {
   return cudaSuccess;
 }
 
-template <int EPI>
+template <int EPI, int BN = 128>
 static void launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
                        long M, int N, int K, int a_cols, const EpiParams& ep, int* err_flag, int num_sms, bool pdl,
                        cudaStream_t s) {
-  const long tiles = ((M + kBM - 1) / kBM) * ((N + 127) / 128);
+  const long tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
   const int grid = (int)(tiles < num_sms ? tiles : num_sms);
-  launch_dependent(gemm_bf16_kernel<128, EPI>, dim3(grid), dim3(kGemmThreads), SmemPlan<128, EPI>::kSmemBytes, s, 1, pdl,
+  launch_dependent(gemm_bf16_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), SmemPlan<BN, EPI>::kSmemBytes, s, 1, pdl,
                    ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag);
 }
 
@@ -991,12 +996,30 @@ void launch_gemm_bf16(const CUtensorMap& ta, const CUtensorMap& tb, const CUtens
   // kSmallTilePenalty for its lower efficiency (it reads shared memory at the full 128 B/clk;
   // measured: a round of small tiles takes ~0.8 of a round of pair tiles).
   if (opt.small_tiles && epi != kEpiConv1 && epi != kEpiConv2 && a_cols == K) {
-    constexpr double kSmallTilePenalty = 1.6;
+    // Estimated time in rounds of tiles, in units of one round of 256 x 256 pair tiles (measured on
+    // the FC1 shape at M = 775: a round of 128 x 128 tiles takes ~0.8 of that, a round of 128 x 256
+    // tiles ~1.25: per K block a CTA takes in 32 / 32 / 48 KB)
+    constexpr double kRound128 = 0.8, kRound256 = 1.25;
     const long t_pair = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + 255) / 256);
     const long t_small = ((M + kBM - 1) / kBM) * ((N + 127) / 128);
+    const long t_wide = ((M + kBM - 1) / kBM) * ((N + 255) / 256);
     const long n_pairs = num_sms / 2;
-    const double r_pair = (double)((t_pair + n_pairs - 1) / n_pairs);
-    const double r_small = (double)((t_small + num_sms - 1) / num_sms) * 0.5 * kSmallTilePenalty;
+    double r_pair = (double)((t_pair + n_pairs - 1) / n_pairs);
+    double r_small = (double)((t_small + num_sms - 1) / num_sms) * kRound128;
+    double r_wide = (double)((t_wide + num_sms - 1) / num_sms) * kRound256;
+    if (opt.tile == 1) r_small = r_wide = 1e30;
+    if (opt.tile == 2) r_pair = r_wide = 1e30;
+    if (opt.tile == 3) r_pair = r_small = 1e30;
+    if (r_wide < r_pair && r_wide < r_small) {
+      switch (epi) {
+        case kEpiBias: launch_one<kEpiBias, 256>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+        case kEpiBiasGelu: launch_one<kEpiBiasGelu, 256>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+        case kEpiLnBias: launch_one<kEpiLnBias, 256>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+        case kEpiLnBiasGelu: launch_one<kEpiLnBiasGelu, 256>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+        default: launch_one<kEpiResidSplit, 256>(ta, tb, tc, tc2, M, N, K, a_cols, ep, err_flag, num_sms, pdl, s); break;
+      }
+      return;
+    }
     if (r_small < r_pair) {
       // so few tiles that half of the SMs or more would idle, and a K range long enough for the
       // hand-over between the CTAs to pay: split every tile's K range over a cluster of 2 or 4 CTAs

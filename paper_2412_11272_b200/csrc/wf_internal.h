@@ -60,6 +60,7 @@ struct EpiParams {
 struct LaunchOpts {
   int pdl;          // launch with programmatic stream serialization (a kernel's set-up overlaps its predecessor's tail)
   int small_tiles;  // GEMMs too small to fill the CTA pairs run 128 x 128 tiles on single CTAs
+  int tile;         // 0: the launcher chooses; 1 / 2 / 3: force 256 x 256 pair tiles / 128 x 128 / 128 x 256 single-CTA tiles
   int split_k;      // ... and, when even those leave half of the SMs idle and K has at least this many 64-wide
                     // blocks, split each tile's K range over a cluster of CTAs (0: never)
 };
